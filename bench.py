@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the elastic-KV attention hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ekv|reference]
+
+One "step" = one pass of the hot path over one batch of the Llama-3-8B-shaped decode workload
+(benchmark configs[1]): ekv_write_kv of the 256 new K/V rows through the slot mapping, then
+ekv_attn_decode (split pass + combine pass) of 256 sequences with context lengths U[1024, 8192]
+whose blocks are randomly permuted over the pool.  value = algorithmic bytes of the step / time.
+Multi-GPU runs are independent replicas (one pool per rank, no collective on the data path).
+
+The JSON line also carries: roofline (decode kernels, timed live with CUDA events), e2e (same
+step through host buffers), cpu_baseline (the CPU oracle on this machine's host cores), and two side
+measurements of the other hot-path rows: prefill-chunk TFLOP/s and grow/shrink ms.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import ekv_inputs as I  # noqa: E402
+
+METRIC = "decode-attn HBM GB/s (% peak); prefill-chunk TFLOP/s (% peak); grow/shrink ms"
+UNIT = "GB/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes (read + write) per launch of the decode split kernel on this workload, from the ncu
+# capture summarised in profiles/decode_split_c2.md (None until a capture exists).
+DECODE_SPLIT_DRAM_TRAFFIC_BYTES = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- workload
+
+
+class DecodeWorkload:
+    """configs[1] resident on one GPU: pool filled by the seeded generator, tables, lengths, inputs."""
+
+    def __init__(self, cfg: I.Config, device: torch.device, batch: int | None = None):
+        import paper_2608_23658_b200 as ekv
+        self.ekv, self.cfg, self.shape, self.dev = ekv, cfg, cfg.shape, device
+        s = cfg.shape
+        self.lengths = I.decode_lengths(cfg, batch)
+        self.B = len(self.lengths)
+        need = int(I.blocks_for(self.lengths, s.block_size).sum())
+        pool_blocks = int(need * 1.1) + 64
+        self.pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim,
+                             base_blocks=pool_blocks, device=device.index or 0)
+        live = self.pool.info.live_blocks
+        self.tables, _ = I.assign_blocks(cfg.seed, 12, self.lengths, s.block_size, live)
+        I.fill_pool_layer_(self.pool.layer_tensor(0), cfg.seed)
+        n_q = self.B * s.num_q_heads * s.head_dim
+        n_kv = self.B * s.num_kv_heads * s.head_dim
+        # host-side (pinned) inputs of one step
+        self.h_q = I.normal_bf16(cfg.seed, 3, 0, n_q).view(self.B, s.num_q_heads, s.head_dim).pin_memory()
+        self.h_k = I.normal_bf16(cfg.seed, 4, 0, n_kv).view(self.B, s.num_kv_heads, s.head_dim).pin_memory()
+        self.h_v = I.normal_bf16(cfg.seed, 5, 0, n_kv).view(self.B, s.num_kv_heads, s.head_dim).pin_memory()
+        self.h_slots = I.last_token_slots(self.lengths, self.tables, s.block_size).pin_memory()
+        self.h_tables = self.tables.pin_memory()
+        self.h_lens = self.lengths.to(torch.int32).pin_memory()
+        self.h_out = torch.empty(self.B, s.num_q_heads, s.head_dim, dtype=torch.bfloat16).pin_memory()
+        # device-resident copies
+        self.q, self.k, self.v = self.h_q.to(device), self.h_k.to(device), self.h_v.to(device)
+        self.slots, self.d_tables, self.d_lens = self.h_slots.to(device), self.h_tables.to(device), self.h_lens.to(device)
+        self.out = torch.empty_like(self.q)
+        self.ws = self.pool.workspace(self.B, int(self.tables.shape[1]) * s.block_size)
+        self.scale = 1.0 / math.sqrt(s.head_dim)
+        self.decode_bytes = I.decode_algorithmic_bytes(self.lengths, s)
+        self.write_bytes = I.write_algorithmic_bytes(self.B, s)
+        torch.cuda.synchronize(device)
+
+    def step_resident(self, ev=None):
+        p = self.pool
+        if ev:
+            ev[0].record()
+        p.write_kv(0, self.k, self.v, self.slots)
+        if ev:
+            ev[1].record()
+        p.attn_decode(0, self.q, self.d_tables, self.d_lens, self.scale, out=self.out, workspace=self.ws)
+        if ev:
+            ev[2].record()
+
+    def step_e2e(self):
+        """Same step through host buffers: pinned H2D of the step's inputs, D2H of the result."""
+        nb = True
+        self.q.copy_(self.h_q, non_blocking=nb)
+        self.k.copy_(self.h_k, non_blocking=nb)
+        self.v.copy_(self.h_v, non_blocking=nb)
+        self.slots.copy_(self.h_slots, non_blocking=nb)
+        self.d_tables.copy_(self.h_tables, non_blocking=nb)
+        self.d_lens.copy_(self.h_lens, non_blocking=nb)
+        self.step_resident()
+        self.h_out.copy_(self.out, non_blocking=nb)
+
+    def e2e_bytes(self):
+        h2d = sum(t.numel() * t.element_size() for t in (self.h_q, self.h_k, self.h_v, self.h_slots, self.h_tables,
+                                                         self.h_lens))
+        return h2d, self.h_out.numel() * self.h_out.element_size()
+
+    def close(self):
+        self.pool.close()
+
+
+def timed_loop(fn, steps, device, dist):
+    """barrier + sync, K steps between two CUDA events on the current stream, sync + barrier; max over ranks."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(device)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize(device)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize(device)
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t[0])
+    return ms
+
+
+# ----------------------------------------------------------------------------- side measurements
+
+
+def measure_prefill(device, peaks, reps=3):
+    """Prefill-chunk TFLOP/s on the configs[2] prompt: 32768 tokens as four 8192-token chunks over
+    cached prefixes 0/8k/16k/24k, and as one 32768-token chunk."""
+    import paper_2608_23658_b200 as ekv
+    cfg, s = I.C3, I.C3.shape
+    Lp = cfg.prompt_len
+    nblk = Lp // s.block_size
+    pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=nblk + 64,
+                    device=device.index or 0)
+    try:
+        live = pool.info.live_blocks
+        table, _ = I.assign_blocks(cfg.seed, 13, torch.tensor([Lp]), s.block_size, live)
+        I.fill_pool_layer_(pool.layer_tensor(0), cfg.seed)
+        q = I.normal_bf16(cfg.seed, 6, 0, Lp * s.num_q_heads * s.head_dim, device=device).view(Lp, s.num_q_heads, s.head_dim)
+        out = torch.empty_like(q)
+        d_table = table.to(device)
+        scale = 1.0 / math.sqrt(s.head_dim)
+        res = {}
+        for chunk in cfg.chunk_lens:
+            calls = []
+            for start in range(0, Lp, chunk):
+                cu = torch.tensor([0, chunk], dtype=torch.int32)
+                calls.append((q[start:start + chunk], out[start:start + chunk], cu.to(device), cu,
+                              torch.tensor([start + chunk], dtype=torch.int32, device=device)))
+
+            def run():
+                for (qq, oo, cud, cuh, sl) in calls:
+                    pool.attn_prefill_chunk(0, qq, d_table, cud, cuh, sl, scale, out=oo)
+            run()
+            torch.cuda.synchronize(device)
+            best = float("inf")
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                run()
+                e1.record()
+                torch.cuda.synchronize(device)
+                best = min(best, e0.elapsed_time(e1))
+            flops = sum(I.prefill_flops(chunk, start, s) for start in range(0, Lp, chunk))
+            tf = flops / (best * 1e-3) / 1e12
+            res[f"chunk_{chunk}"] = {"ms": round(best, 3), "tflops": round(tf, 1),
+                                     "frac_of_measured_bf16": round(tf / peaks["bf16_tflops"], 4),
+                                     "frac_of_nominal_2250": round(tf / 2250.0, 4)}
+        res["workload"] = "c3 prompt 32768 tokens, 32/8 heads d128, causal-exact FLOPs of both contractions"
+        return res
+    finally:
+        pool.close()
+
+
+def measure_toggle(device, cycles=5):
+    """grow / shrink ms on the configs[4] geometry: 32 layers x 96 MiB elastic (3 GiB reserve)."""
+    import paper_2608_23658_b200 as ekv
+    cfg, s = I.C5, I.C5.shape
+    per_layer = cfg.elastic_total_bytes // cfg.num_layers
+    pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=512,
+                    elastic_blocks=per_layer // s.block_bytes, num_layers=cfg.num_layers, device=device.index or 0)
+    try:
+        rows = {"grow_release": [], "shrink_release": [], "grow_keep": [], "shrink_keep": []}
+        for _ in range(cycles):
+            rows["grow_release"].append(pool.grow())
+            rows["shrink_release"].append(pool.shrink())
+        pool.grow()
+        for _ in range(cycles):
+            rows["shrink_keep"].append(pool.shrink(keep_physical=True))
+            rows["grow_keep"].append(pool.grow())
+        out = {k: {"driver_ms_median": round(statistics.median(r[0] for r in v), 3),
+                   "call_ms_median": round(statistics.median(r[1] for r in v), 3),
+                   "call_ms_max": round(max(r[1] for r in v), 3)} for k, v in rows.items()}
+        out["workload"] = f"{cfg.num_layers} layers x {per_layer >> 20} MiB elastic, {cycles} cycles per mode"
+        out["paper_a100_context_ms"] = {"decommit": 3.0, "commit": 30.0, "naive_commit": 180.0}
+        return out
+    finally:
+        pool.close()
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+
+
+def oracle_decode_sample(cfg, max_seqs=24):
+    """Times the CPU oracle, as it stands, on a bounded sample of the decode workload."""
+    import oracle
+    s = cfg.shape
+    lengths = I.decode_lengths(cfg)
+    need = int(I.blocks_for(lengths, s.block_size).sum())
+    tables, _ = I.assign_blocks(cfg.seed, 12, lengths, s.block_size, int(need * 1.1) + 64)
+    ids = list(range(min(max_seqs, len(lengths))))
+    cache, ctab, clen = I.compact_host_cache(cfg.seed, 0, tables, lengths, ids, s)
+    q = I.normal_bf16(cfg.seed, 3, 0, len(lengths) * s.num_q_heads * s.head_dim).view(len(lengths), s.num_q_heads, s.head_dim)
+    qs = q[ids].contiguous()
+    scale = 1.0 / math.sqrt(s.head_dim)
+    oracle.attn_decode(cache, s.num_q_heads, s.num_kv_heads, s.block_size, s.head_dim, qs[:1], ctab[:1], clen[:1], scale)
+    nbytes = I.decode_algorithmic_bytes(clen, s)
+
+    def one():
+        t0 = time.perf_counter()
+        oracle.attn_decode(cache, s.num_q_heads, s.num_kv_heads, s.block_size, s.head_dim, qs, ctab, clen, scale)
+        return time.perf_counter() - t0
+    return one, nbytes, f"{len(ids)} of {len(lengths)} sequences of the workload ({int(clen.sum())} cached tokens, all heads)", \
+        oracle.threads()
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = I.C2
+    one, nbytes, sample, cores = oracle_decode_sample(cfg)
+    for _ in range(args.warmup):
+        one()
+    times = [one() for _ in range(args.steps)]
+    total = sum(times)
+    value = nbytes * args.steps / total / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(1e3 * total / args.steps, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "sample": sample},
+            "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- main
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ekv", choices=["ekv", "reference"])
+    ap.add_argument("--batch", type=int, default=None, help="debug: fewer sequences than the named workload")
+    ap.add_argument("--no-extras", action="store_true", help="skip prefill / toggle / cpu_baseline side measurements")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the ekv path has no CPU fallback (use --impl reference for the oracle)")
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=device)
+        dist = dist_mod
+
+    peaks, peaks_kind = measured_peaks()
+    cfg = I.C2
+    wl = DecodeWorkload(cfg, device, args.batch)
+    assert wl.decode_bytes > 200e6 or args.batch, "working set must exceed L2"
+
+    for _ in range(args.warmup):
+        wl.step_resident()
+    # per-step kernel-group durations, measured live inside the timed region
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    it = iter(evs)
+    with ClockSampler(device.index or 0) as clk:
+        ms = timed_loop(lambda: wl.step_resident(next(it)), args.steps, device, dist)
+    clocks = clk.summary()
+    write_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    decode_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    st = wl.pool.poll_status()
+    if st != 0:
+        raise SystemExit(f"bench.py: device status {st!r} after the timed region")
+
+    for _ in range(args.warmup):
+        wl.step_e2e()
+    ms_e2e = timed_loop(wl.step_e2e, args.steps, device, dist)
+
+    step_bytes = wl.decode_bytes + wl.write_bytes
+    value = world * step_bytes * args.steps / (ms * 1e-3) / 1e9
+    e2e_value = world * step_bytes * args.steps / (ms_e2e * 1e-3) / 1e9
+    achieved = wl.decode_bytes / (decode_ms * 1e-3) / 1e9
+    h2d, d2h = wl.e2e_bytes()
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": wl.B, "heads": "32q/8kv", "head_dim": 128, "block_size": 16,
+                   "context_tokens": int(wl.lengths.sum()), "step": "ekv_write_kv + ekv_attn_decode (split + combine)",
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (%.2f GB of KV per step)" % (wl.decode_bytes / 1e9)},
+        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel<128> + decode_combine_kernel<128>",
+                     "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(achieved / peaks["hbm_gbs"], 4), "peak_kind": f"{peaks_kind} copy bandwidth",
+                     "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": DECODE_SPLIT_DRAM_TRAFFIC_BYTES,
+                     "algorithmic_bytes_per_launch": wl.decode_bytes, "launch_ms": round(decode_ms, 4),
+                     "write_kv_ms": round(write_ms, 4)},
+        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": round(ms_e2e / args.steps, 4)},
+        "gpu_launches": 3 * args.steps,
+        "clocks": clocks,
+    }
+    wl.close()
+    if rank == 0 and world == 1 and not args.no_extras:
+        torch.cuda.empty_cache()
+        line["prefill"] = measure_prefill(device, peaks)
+        torch.cuda.empty_cache()
+        line["toggle"] = measure_toggle(device)
+        one, nbytes, sample, cores = oracle_decode_sample(cfg)
+        one()
+        reps, t = 0, 0.0
+        while t < 10.0 and reps < 60:
+            t += one()
+            reps += 1
+        line["cpu_baseline"] = {"value": round(nbytes * reps / t / 1e9, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{sample}, {reps} passes"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -205,3 +205,57 @@ CONFIGS = {c.name: c for c in (C1, C2, C3, C4, C5)}
 def decode_lengths(cfg: Config, batch: int | None = None) -> torch.Tensor:
     d = cfg.decode
     return uniform_ints(cfg.seed, 11, d.batch if batch is None else batch, d.len_lo, d.len_hi)
+
+
+# ------------------------------------------------------------------ physical fills and host mirrors
+
+KV_STREAM = 21  # stream id of "pool content as a function of the physical element index"
+
+
+def fill_pool_layer_(layer_view: torch.Tensor, seed: int, layer: int = 0, first_block: int = 0) -> None:
+    """Fill a [blocks, 2, Hkv, bs, d] bf16 view of a layer (starting at physical block first_block)
+    so that element e of the layer holds normal_bf16(seed, KV_STREAM + layer, e)."""
+    block_elems = layer_view[0].numel()
+    fill_normal_bf16_(layer_view, seed, KV_STREAM + layer, start=first_block * block_elems)
+
+
+def host_blocks(seed: int, layer: int, block_ids, block_elems: int) -> torch.Tensor:
+    """CPU regeneration of the listed physical blocks of a fill_pool_layer_ pool: bf16 [n, block_elems]."""
+    out = torch.empty(len(block_ids), block_elems, dtype=torch.bfloat16)
+    for i, n in enumerate(block_ids):
+        out[i] = normal_bf16(seed, KV_STREAM + layer, int(n) * block_elems, block_elems)
+    return out
+
+
+def compact_host_cache(seed: int, layer: int, tables: torch.Tensor, lengths: torch.Tensor, seq_ids, shape: Shape):
+    """Host mirror holding only the blocks of the listed sequences, renumbered 0..n-1.
+    Returns (cache bf16 [n*block_elems], compact tables int32 [len(seq_ids), width], lengths)."""
+    nb = blocks_for(lengths, shape.block_size)
+    width = int(nb[list(seq_ids)].max())
+    ctab = torch.full((len(seq_ids), width), -1, dtype=torch.int32)
+    ids = []
+    for i, b in enumerate(seq_ids):
+        n = int(nb[b])
+        ctab[i, :n] = torch.arange(len(ids), len(ids) + n, dtype=torch.int32)
+        ids += tables[b, :n].tolist()
+    cache = host_blocks(seed, layer, ids, shape.block_elems).view(-1)
+    return cache, ctab, lengths[list(seq_ids)].clone()
+
+
+def decode_algorithmic_bytes(lengths: torch.Tensor, shape: Shape) -> int:
+    """Bytes a decode step must move: every cached K and V element once, Q in, O out, block table."""
+    B = len(lengths)
+    kv = int(lengths.sum()) * shape.token_bytes
+    qo = 2 * B * shape.num_q_heads * shape.head_dim * 2
+    table = int(blocks_for(lengths, shape.block_size).sum()) * 4
+    return kv + qo + table
+
+
+def write_algorithmic_bytes(T: int, shape: Shape) -> int:
+    return 2 * T * shape.token_bytes + 8 * T
+
+
+def prefill_flops(chunk: int, prefix: int, shape: Shape) -> int:
+    """Causal-exact FLOPs of both contractions: 4*d*Hq per (query row, visible key) pair."""
+    pairs = chunk * prefix + chunk * (chunk + 1) // 2
+    return 4 * shape.head_dim * shape.num_q_heads * pairs

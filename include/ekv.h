@@ -1,0 +1,238 @@
+/*
+ * ekv.h -- C ABI of libekv: attention over a block-indexed KV cache that lives in ONE
+ * contiguous virtual address range per layer, backed by a base handle plus an elastic handle.
+ *
+ * The calls follow the paper's statement of the problem (section "An Elastic KV Mechanism"):
+ *   - "Two handles, one virtual range": reserve one range per layer sized base + elastic, keep
+ *     the base handle always mapped, map / unmap the elastic handle at the TOP of the range,
+ *     aligned to the VMM granularity                        -> ekv_pool_create, ekv_grow, ekv_shrink
+ *   - "The contiguity constraint": the attention kernel indexes the layer's tensor by block id
+ *     through one base pointer, so the kernels never change when the elastic slice comes or
+ *     goes                                                  -> ekv_write_kv, ekv_attn_decode,
+ *                                                              ekv_attn_prefill_chunk
+ *   - "Controller": committing admits the top block ids, decommitting drains, syncs, unmaps
+ *                                                           -> the live-block limit and ordering
+ *                                                              rules of ekv_grow / ekv_shrink
+ *
+ * General rules
+ *   - Every call returns an ekv_status_t and never throws.  Argument errors are detected on the
+ *     host before any state changes.  ekv_last_error() gives a one-line detail for the calling
+ *     thread's most recent failure.
+ *   - Pointers marked DEVICE are device addresses owned by the caller (any allocator); pointers
+ *     marked HOST are ordinary host memory.  The pool owns the KV ranges and physical handles.
+ *   - ekv_write_kv / ekv_attn_* are asynchronous: they enqueue work on `stream` (a cudaStream_t /
+ *     CUstream passed as void*, NULL = legacy default stream) and return without synchronising.
+ *   - ekv_grow / ekv_shrink are host-synchronous and must not run concurrently with any other
+ *     call on the same pool (the caller serialises them at a step boundary).
+ *   - There is no CPU fallback: without a CUDA device every compute call fails with EKV_ERR_CUDA.
+ *
+ * KV layout (part of the boundary).  All layers share one geometry.  From ekv_layer_ptr(layer),
+ * channel x of token-in-block t of kv-head h of the K (kv=0) or V (kv=1) half of physical block n
+ * is the bf16 at byte offset
+ *       ((((n*2 + kv)*num_kv_heads + h)*block_size + t)*head_dim + x) * 2 .
+ * Block n therefore occupies bytes [n*block_bytes, (n+1)*block_bytes); blocks 0..base_blocks-1
+ * are backed by the base handle, blocks base_blocks..base_blocks+elastic_blocks-1 by the elastic
+ * handle.  A slot is block*block_size + t.
+ */
+#ifndef EKV_H_
+#define EKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define EKV_API __attribute__((visibility("default")))
+#else
+#define EKV_API
+#endif
+
+typedef struct ekv_pool ekv_pool_t; /* opaque */
+
+typedef enum ekv_status {
+    EKV_OK = 0,
+    EKV_ERR_INVALID = 1,   /* bad argument; nothing changed */
+    EKV_ERR_CUDA = 2,      /* a CUDA runtime / driver call failed, or no device / driver */
+    EKV_ERR_OOM = 3,       /* physical memory could not be created; pool left in its prior state */
+    EKV_ERR_STATE = 4,     /* e.g. grow when grown, shrink when shrunk, compute on a host-only pool */
+    EKV_ERR_BLOCK_OOB = 5, /* latched by a kernel: a block id or slot was outside [0, live_blocks) */
+    EKV_ERR_TIMEOUT = 6,   /* latched by a kernel: a bounded wait on a copy barrier ran out */
+    EKV_ERR_WORKSPACE = 7  /* workspace missing, misaligned (256 B) or too small */
+} ekv_status_t;
+
+enum { EKV_BF16 = 0 };
+
+/* flag bits */
+enum {
+    EKV_START_GROWN = 1u << 0,   /* ekv_pool_create: map the elastic slice right away */
+    EKV_KEEP_PHYSICAL = 1u << 1  /* ekv_shrink: unmap only, keep the elastic handle (bytes survive
+                                    until the next ekv_grow maps it again) */
+};
+
+typedef struct ekv_pool_desc {
+    int32_t device;         /* CUDA device ordinal */
+    int32_t num_layers;     /* >= 1 */
+    int32_t num_q_heads;    /* multiple of num_kv_heads; group = num_q_heads/num_kv_heads in 1..8 */
+    int32_t num_kv_heads;
+    int32_t head_dim;       /* 64 or 128 */
+    int32_t block_size;     /* 16 */
+    int32_t dtype;          /* EKV_BF16 */
+    uint32_t flags;         /* EKV_START_GROWN */
+    int64_t base_blocks;    /* per layer, >= 1; rounded UP to whole granules */
+    int64_t elastic_blocks; /* per layer, >= 0; rounded UP to whole granules */
+} ekv_pool_desc_t;
+
+typedef struct ekv_pool_info {
+    uint64_t granularity;    /* VMM minimum allocation granularity in bytes (2 MiB in the paper) */
+    uint64_t block_bytes;    /* 2*num_kv_heads*block_size*head_dim*2 */
+    uint64_t base_bytes;     /* per layer, after rounding */
+    uint64_t elastic_bytes;  /* per layer, after rounding */
+    int64_t base_blocks;     /* after rounding */
+    int64_t elastic_blocks;  /* after rounding */
+    int64_t live_blocks;     /* base_blocks, or base_blocks + elastic_blocks while grown */
+    int32_t grown;           /* elastic slice mapped */
+    int32_t physical_held;   /* elastic handles exist (mapped, or kept by EKV_KEEP_PHYSICAL) */
+    int32_t num_layers;
+    int32_t reserved;
+} ekv_pool_info_t;
+
+/*
+ * ekv_pool_create -- "Two handles, one virtual range".  Per layer: reserve a virtual range of
+ * (base+elastic) bytes, create + map + grant the base handle; the elastic sub-range stays unmapped
+ * unless EKV_START_GROWN.  Sizes are rounded up to the allocation granularity, which must be a
+ * multiple of block_bytes.  desc, out: HOST.  On failure nothing is left allocated.
+ */
+EKV_API ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out);
+
+/* Unmaps and releases everything the pool owns.  The caller must have synchronised all streams
+ * that used the pool.  NULL is accepted. */
+EKV_API ekv_status_t ekv_pool_destroy(ekv_pool_t *pool);
+
+/* Geometry and state after rounding.  info: HOST. */
+EKV_API ekv_status_t ekv_pool_info(const ekv_pool_t *pool, ekv_pool_info_t *info);
+
+/* Device address of the layer's range; constant for the pool's life whether the elastic slice is
+ * mapped or not (the paper's "the virtual range never moves").  dptr: HOST, receives a DEVICE
+ * address.  Touching bytes of the elastic sub-range while it is unmapped faults the context. */
+EKV_API ekv_status_t ekv_layer_ptr(const ekv_pool_t *pool, int32_t layer, void **dptr);
+
+/*
+ * ekv_grow -- commit ("Toggle cost", "Controller"): for every layer create the elastic handle if
+ * it is not held, map it at the top of the range, grant access; then raise the device-side live
+ * limit to base+elastic on `stream`.  Elastic bytes are undefined after a grow that had to create
+ * the handle.  If creation or mapping fails at any layer, everything this call mapped or created
+ * is undone, the pool stays shrunk and EKV_ERR_OOM / EKV_ERR_CUDA is returned.
+ * ms_out (HOST, may be NULL) receives ms_out[0] = host time of the driver calls alone and
+ * ms_out[1] = host time of the whole call including stream synchronisation.
+ */
+EKV_API ekv_status_t ekv_grow(ekv_pool_t *pool, void *stream, uint32_t flags, double *ms_out);
+
+/*
+ * ekv_shrink -- decommit ("Controller": drain, sync, unmap).  Lowers the live limit to base_blocks
+ * on `stream`, synchronises the whole device (every stream that may still read elastic blocks),
+ * unmaps the elastic sub-range of every layer and, unless EKV_KEEP_PHYSICAL, releases the
+ * handles (the memory returns to the driver).  Precondition the library cannot check: the caller
+ * no longer uses block ids >= base_blocks ("drains those blocks").  A kernel launched afterwards
+ * with such an id skips it and latches EKV_ERR_BLOCK_OOB instead of faulting.  ms_out as above.
+ */
+EKV_API ekv_status_t ekv_shrink(ekv_pool_t *pool, void *stream, uint32_t flags, double *ms_out);
+
+/*
+ * ekv_write_kv -- slot-mapped KV write into the paged pool (section "Background and Motivation",
+ * "KV allocation in vLLM": fixed-size blocks handed to requests).  An exact scatter of bit
+ * patterns: token i's k[i,h,:] and v[i,h,:] go to slot slot_mapping[i] of `layer`.
+ * k, v: DEVICE, bf16 [T, num_kv_heads, head_dim], contiguous, 16-byte aligned.
+ * slot_mapping: DEVICE int64 [T]; negative = skip the token; a slot whose block is >= the live
+ * limit is skipped and latches EKV_ERR_BLOCK_OOB.  Duplicate slots in one call: unspecified
+ * winner.  T == 0 is a no-op.
+ */
+EKV_API ekv_status_t ekv_write_kv(ekv_pool_t *pool, int32_t layer, const void *k, const void *v,
+                          const int64_t *slot_mapping, int32_t T, void *stream);
+
+/* Bytes of scratch ekv_attn_decode needs for any call with B <= max_batch and
+ * max_blocks_per_seq*block_size <= max_seq_len (rounded up to a block).  ekv_attn_prefill_chunk
+ * needs none.  Returns 0 for a NULL pool. */
+EKV_API size_t ekv_attn_workspace_bytes(const ekv_pool_t *pool, int32_t max_batch, int32_t max_seq_len);
+
+/*
+ * ekv_attn_decode -- grouped-query attention of ONE query token per sequence over that sequence's
+ * cached keys/values ("the attention kernel" of "The contiguity constraint"; decode contributes
+ * one token per sequence per step, "Why the penalty is small").
+ *   out[b,h,:] = sum_j softmax_j(scale * q[b,h,:].K_j) V_j ,  j = 0 .. seq_lens[b]-1,
+ * where key j of sequence b is token j%block_size of block block_tables[b][j/block_size] and query
+ * head h reads kv-head h/(num_q_heads/num_kv_heads).  seq_lens[b] includes the query token (its
+ * K/V were written first).  bf16 in, fp32 accumulate, bf16 out (round to nearest even).
+ * q, out: DEVICE bf16 [B, num_q_heads, head_dim], 16-byte aligned.
+ * block_tables: DEVICE int32 [B, max_blocks_per_seq]; entries at or past ceil(seq_len/block_size)
+ * are never read.  seq_lens: DEVICE int32 [B]; 0 gives a zero row; values above
+ * max_blocks_per_seq*block_size are clamped to it.
+ * workspace: DEVICE, 256-byte aligned, >= ekv_attn_workspace_bytes(pool, B, max_blocks_per_seq*
+ * block_size); contents need no initialisation; calls that share it must be stream-ordered.
+ * Two passes: a split pass over fixed-size key ranges writing fp32 partials, and a combine pass.
+ * The split plan depends only on (B, max_blocks_per_seq), so results are bitwise reproducible and
+ * independent of which physical blocks hold the data.
+ */
+EKV_API ekv_status_t ekv_attn_decode(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
+                             const int32_t *block_tables, int32_t max_blocks_per_seq,
+                             const int32_t *seq_lens, int32_t B, float scale, void *workspace,
+                             size_t workspace_bytes, void *stream);
+
+/*
+ * ekv_attn_prefill_chunk -- causal attention of a prompt chunk over its cached prefix plus itself
+ * (chunked prefill: "The Decisive Test", "Why the penalty is small": chunking splits the same
+ * work across steps).  Request r owns query rows cu_q_lens[r] .. cu_q_lens[r+1]-1 (c_r rows) and
+ * seq_lens[r] = prefix_r + c_r keys; row i of the chunk sits at absolute position prefix_r + i and
+ * attends to keys 0 .. prefix_r + i.  All keys/values, the chunk's own included, are read from
+ * the cache (run ekv_write_kv for the chunk first).
+ * q, out: DEVICE bf16 [T, num_q_heads, head_dim], 16-byte aligned, T = cu_q_lens[R].
+ * block_tables: DEVICE int32 [R, max_blocks_per_seq].  seq_lens: DEVICE int32 [R].
+ * cu_q_lens: DEVICE int32 [R+1], non-decreasing, cu_q_lens[0] = 0.
+ * cu_q_lens_host: HOST copy of the same R+1 values (used to size the launch without a sync).
+ * Requests with seq_lens[r] < c_r are invalid (rows produce zeros, EKV_ERR_BLOCK_OOB is latched).
+ */
+EKV_API ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
+                                    const int32_t *block_tables, int32_t max_blocks_per_seq,
+                                    const int32_t *cu_q_lens, const int32_t *cu_q_lens_host,
+                                    const int32_t *seq_lens, int32_t R, float scale, void *stream);
+
+/* Non-blocking read-and-clear of the status latched by kernels (EKV_OK, EKV_ERR_BLOCK_OOB or
+ * EKV_ERR_TIMEOUT; the latter wins).  Meaningful after the launching stream was synchronised. */
+EKV_API ekv_status_t ekv_poll_status(ekv_pool_t *pool);
+
+EKV_API const char *ekv_status_string(ekv_status_t status);
+
+/* One-line description of the calling thread's most recent failing call ("" if none). */
+EKV_API const char *ekv_last_error(void);
+
+/*
+ * Virtual-memory backend.  The pool's state machine (rounding, create / grow / shrink / destroy,
+ * unwinding after a failure) talks to the driver only through this table.  The default table
+ * calls the CUDA driver VMM API (cuMemAddressReserve, cuMemCreate, cuMemMap, cuMemSetAccess,
+ * cuMemUnmap, cuMemRelease, cuMemAddressFree, cuMemGetAllocationGranularity).  Installing another
+ * table lets the state machine be exercised on a host without a GPU; pools created while a
+ * replacement table is installed are host-only: they hold no device state and every compute call
+ * on them returns EKV_ERR_STATE.  Each function returns 0 on success, 2 for out-of-memory, any
+ * other value for failure.  ekv_set_vmm_backend(NULL) restores the default; it must not be
+ * called while pools exist.
+ */
+typedef struct ekv_vmm_backend {
+    void *user;
+    int (*granularity)(void *user, int device, uint64_t *bytes);
+    int (*reserve)(void *user, uint64_t size, uint64_t alignment, uint64_t *va);
+    int (*unreserve)(void *user, uint64_t va, uint64_t size);
+    int (*create)(void *user, uint64_t size, int device, uint64_t *handle);
+    int (*release)(void *user, uint64_t handle);
+    int (*map)(void *user, uint64_t va, uint64_t size, uint64_t handle);
+    int (*unmap)(void *user, uint64_t va, uint64_t size);
+    int (*set_access)(void *user, uint64_t va, uint64_t size, int device);
+} ekv_vmm_backend_t;
+
+EKV_API ekv_status_t ekv_set_vmm_backend(const ekv_vmm_backend_t *backend);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EKV_H_ */

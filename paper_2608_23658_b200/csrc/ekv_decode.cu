@@ -1,0 +1,396 @@
+// ekv_attn_decode: GQA decode attention over the block-indexed KV range, HBM-bandwidth bound.
+//
+// Split pass.  One CTA per (sequence, kv-head, key range of `chunk_tokens`).  Each of the 4 warps
+// owns every 4th 16-token block of the range and its own ring of shared-memory stages; lane 0
+// feeds the ring with TMA tile loads (one 64-channel x 16-token box per 2 KiB, 128-byte swizzle)
+// that complete on per-stage mbarriers, so ~24 KiB per warp can be in flight with no register
+// cost.  The whole query group (<= 8 heads) of the kv-head is processed against each K/V tile,
+// so KV bytes are read from HBM exactly once:
+//     S^T-free formulation on the warp-level tensor path (M is tiny, tcgen05 does not apply):
+//       S[head, token]  = Q[head, :] . K[token, :]      mma m16n8k16, heads padded to 16 rows
+//       O^T[d, head]   += V^T[d, token] P^T[token, head] mma m16n8k16, V via ldmatrix.trans
+//     The C fragment of S is exactly the B fragment P^T needs, so no shuffle sits between them.
+// Online softmax keeps a running max per head (quad shuffles) in the exp2 domain.  The 4 warps
+// merge through shared memory and write one fp32 partial (m, l, o[d]) per (sequence, head, split).
+//
+// Combine pass.  One CTA per (sequence, q-head): log-sum-exp merge of the partials -> bf16.
+//
+// The plan (chunk_tokens) depends only on the call's shape arguments and the summation order only
+// on logical key positions, so results are bitwise reproducible and independent of which physical
+// blocks (base or elastic) hold the data.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "ekv_internal.h"
+#include "ptx.cuh"
+
+namespace ekv {
+
+static constexpr int kDecodeWarps = 4;
+static constexpr int kDecodeStages = 3;
+static constexpr int kBoxBytes = 16 * 128;  // 16 tokens x 64 bf16 channels
+static constexpr int kChunkMaxLimit = 2048; // 32 blocks per warp: one block id per lane
+
+struct DecodeParams {
+    const __nv_bfloat16 *q;
+    const int *block_tables;
+    const int *seq_lens;
+    const long long *live;
+    unsigned *status;
+    float *part_o;   // [B*Hq*nsplit, D]
+    float2 *part_ml; // [B*Hq*nsplit]
+    __nv_bfloat16 *out;
+    int max_blocks, num_q_heads, num_kv_heads, group;
+    int chunk_tokens, nsplit;
+    float scale_log2;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kDecodeWarps * 32, 2)
+decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const DecodeParams p) {
+    constexpr int BOXES = D / 64;
+    constexpr int TILE_BYTES = BOXES * kBoxBytes;
+    constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+    constexpr int KSTEPS = D / 16;
+    constexpr unsigned FULL = 0xffffffffu;
+
+    const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = lane >> 2, c = lane & 3;
+
+    int L = p.seq_lens[b];
+    L = max(0, min(L, p.max_blocks * 16));
+    const int t_begin = split * p.chunk_tokens;
+    if (t_begin >= L) return;  // whole CTA leaves before any barrier exists
+    const int t_end = min(L, t_begin + p.chunk_tokens);
+    const int nblk = (t_end - t_begin + 15) >> 4;
+    const int nw = max(0, (nblk - warp + kDecodeWarps - 1) / kDecodeWarps);  // blocks this warp owns (<= 32)
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_u32 = smem_u32(smem_raw);
+    const uint32_t base_u32 = (raw_u32 + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base_u32 - raw_u32);
+    const uint32_t my_stages = base_u32 + warp * kDecodeStages * STAGE_BYTES;
+    const uint32_t my_bars = base_u32 + kDecodeWarps * kDecodeStages * STAGE_BYTES + warp * kDecodeStages * 8;
+
+    if (lane == 0) {
+        prefetch_tensormap(&kvmap);
+        for (int s = 0; s < kDecodeStages; ++s) mbar_init(my_bars + 8 * s, 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
+
+    // Block ids of this warp's blocks: lane i holds the id of its i-th block.
+    const long long live = *p.live;
+    const int *bt = p.block_tables + (size_t)b * p.max_blocks + (t_begin >> 4) + warp;
+    int my_id = (lane < nw) ? bt[lane * kDecodeWarps] : 0;
+    const bool my_ok = (lane < nw) && my_id >= 0 && (long long)my_id < live;
+    const unsigned valid_mask = __ballot_sync(FULL, my_ok);
+    if (lane < nw && !my_ok) atomicOr(p.status, EKV_DEV_FLAG_OOB);
+
+    const uint64_t policy = policy_evict_first();
+    auto issue = [&](int i) {
+        const int id = __shfl_sync(FULL, my_id, i);
+        if (lane == 0 && ((valid_mask >> i) & 1u)) {
+            const int stage = i % kDecodeStages;
+            const uint32_t bar = my_bars + 8 * stage;
+            const uint32_t dst = my_stages + stage * STAGE_BYTES;
+            const int row_k = (id * 2 * p.num_kv_heads + g) * 16;
+            const int row_v = row_k + p.num_kv_heads * 16;
+            mbar_expect_tx(bar, STAGE_BYTES);
+#pragma unroll
+            for (int x = 0; x < BOXES; ++x) {
+                tma_load_2d_hint(dst + x * kBoxBytes, &kvmap, 64 * x, row_k, bar, policy);
+                tma_load_2d_hint(dst + TILE_BYTES + x * kBoxBytes, &kvmap, 64 * x, row_v, bar, policy);
+            }
+        }
+    };
+    for (int s = 0; s < kDecodeStages && s < nw; ++s) issue(s);
+
+    // Q fragments (A operand): rows = heads of the group (r < group), zero above.
+    uint32_t qa[KSTEPS][2];
+    {
+        const __nv_bfloat16 *qrow = p.q + ((size_t)b * p.num_q_heads + (size_t)g * p.group + r) * D;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            qa[ks][0] = (r < p.group) ? *reinterpret_cast<const uint32_t *>(qrow + 16 * ks + 2 * c) : 0u;
+            qa[ks][1] = (r < p.group) ? *reinterpret_cast<const uint32_t *>(qrow + 16 * ks + 8 + 2 * c) : 0u;
+        }
+    }
+
+    // ldmatrix lane addressing inside one swizzled tile: matrix mi = lane/8, row rr = lane%8.
+    const int mi = lane >> 3, rr = lane & 7;
+    const uint32_t lane_row_off = (8 * (mi >> 1) + rr) * 128;
+    const int lane_par = mi & 1;
+
+    float o[KSTEPS][4];
+#pragma unroll
+    for (int mt = 0; mt < KSTEPS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool failed = false;
+
+    int i = 0;
+    for (; i < nw; ++i) {
+        const int stage = i % kDecodeStages;
+        if ((valid_mask >> i) & 1u) {
+            const bool got = mbar_wait(my_bars + 8 * stage, (uint32_t)((i / kDecodeStages) & 1));
+            if (__any_sync(FULL, !got)) {
+                failed = true;
+                break;
+            }
+            const uint32_t kbase = my_stages + stage * STAGE_BYTES;
+            const uint32_t vbase = kbase + TILE_BYTES;
+            const int tok0 = t_begin + (warp + kDecodeWarps * i) * 16;
+            const bool partial = tok0 + 16 > L;
+
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                const int chunk = 2 * ks + lane_par;
+                const uint32_t addr = kbase + (chunk >> 3) * kBoxBytes + lane_row_off + (((chunk & 7) ^ rr) << 4);
+                uint32_t k0, k1, k2, k3;
+                ldmatrix_x4(addr, k0, k1, k2, k3);
+                mma_bf16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, k0, k1);
+                mma_bf16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, k2, k3);
+            }
+            float x0 = s0[0] * p.scale_log2, x1 = s0[1] * p.scale_log2;
+            float x2 = s1[0] * p.scale_log2, x3 = s1[1] * p.scale_log2;
+            uint32_t mask_lo = 0xffffffffu, mask_hi = 0xffffffffu;
+            if (partial) {
+                const int t = tok0 + 2 * c;
+                if (t >= L) x0 = -INFINITY;
+                if (t + 1 >= L) x1 = -INFINITY;
+                if (t + 8 >= L) x2 = -INFINITY;
+                if (t + 9 >= L) x3 = -INFINITY;
+                mask_lo = (t < L ? 0x0000ffffu : 0u) | (t + 1 < L ? 0xffff0000u : 0u);
+                mask_hi = (t + 8 < L ? 0x0000ffffu : 0u) | (t + 9 < L ? 0xffff0000u : 0u);
+            }
+            float mx = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
+            mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 2));
+            const float m_new = fmaxf(m_run, mx);  // finite: token tok0 < L is never masked
+            const float alpha = fast_exp2(m_run - m_new);
+            const float p0 = fast_exp2(x0 - m_new), p1 = fast_exp2(x1 - m_new);
+            const float p2 = fast_exp2(x2 - m_new), p3 = fast_exp2(x3 - m_new);
+            l_run = l_run * alpha + ((p0 + p1) + (p2 + p3));
+            m_run = m_new;
+            if (__any_sync(FULL, alpha != 1.f)) {
+                const float a_lo = __shfl_sync(FULL, alpha, 8 * c);
+                const float a_hi = __shfl_sync(FULL, alpha, 8 * c + 4);
+#pragma unroll
+                for (int mt = 0; mt < KSTEPS; ++mt) {
+                    o[mt][0] *= a_lo;
+                    o[mt][1] *= a_hi;
+                    o[mt][2] *= a_lo;
+                    o[mt][3] *= a_hi;
+                }
+            }
+            const uint32_t pb0 = pack_bf16x2(p0, p1), pb1 = pack_bf16x2(p2, p3);
+#pragma unroll
+            for (int mt = 0; mt < KSTEPS; ++mt) {
+                const int chunk = 2 * mt + lane_par;
+                const uint32_t addr = vbase + (chunk >> 3) * kBoxBytes + lane_row_off + (((chunk & 7) ^ rr) << 4);
+                uint32_t v0, v1, v2, v3;
+                ldmatrix_x4_trans(addr, v0, v1, v2, v3);
+                if (partial) {  // unwritten slots may hold NaN patterns: 0 * NaN must not reach O
+                    v0 &= mask_lo;
+                    v1 &= mask_lo;
+                    v2 &= mask_hi;
+                    v3 &= mask_hi;
+                }
+                mma_bf16_16816(o[mt], v0, v1, v2, v3, pb0, pb1);
+            }
+        }
+        __syncwarp();  // every lane is done reading the stage before it is refilled
+        if (i + kDecodeStages < nw) issue(i + kDecodeStages);
+    }
+
+    if (failed) {
+        // A copy barrier never completed.  Latch the error, give copies still in flight a bounded
+        // chance to land (their destination must stay allocated), and contribute nothing.
+        if (lane == 0) atomicOr(p.status, EKV_DEV_FLAG_TIMEOUT);
+        for (int j = i; j < nw && j < i + kDecodeStages; ++j)
+            if ((valid_mask >> j) & 1u)
+                (void)mbar_wait(my_bars + 8 * (j % kDecodeStages), (uint32_t)((j / kDecodeStages) & 1), 200000000ull);
+        m_run = -INFINITY;
+        l_run = 0.f;
+#pragma unroll
+        for (int mt = 0; mt < KSTEPS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+    }
+
+    l_run += __shfl_xor_sync(FULL, l_run, 1);
+    l_run += __shfl_xor_sync(FULL, l_run, 2);
+
+    // Merge the 4 warps through shared memory (each warp reuses its own, now idle, first stage).
+    float *wo = reinterpret_cast<float *>(base_ptr + warp * kDecodeStages * STAGE_BYTES);  // [8][D]
+    float *wm = wo + 8 * D;                                                                // [8] m, [8] l
+#pragma unroll
+    for (int mt = 0; mt < KSTEPS; ++mt) {
+        wo[(2 * c) * D + 16 * mt + r] = o[mt][0];
+        wo[(2 * c + 1) * D + 16 * mt + r] = o[mt][1];
+        wo[(2 * c) * D + 16 * mt + 8 + r] = o[mt][2];
+        wo[(2 * c + 1) * D + 16 * mt + 8 + r] = o[mt][3];
+    }
+    if (c == 0) {
+        wm[r] = m_run;
+        wm[8 + r] = l_run;
+    }
+    __syncthreads();
+
+    for (int e = threadIdx.x; e < p.group * D; e += kDecodeWarps * 32) {
+        const int h = e / D, x = e % D;
+        float mw[kDecodeWarps], mstar = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kDecodeWarps; ++w) {
+            mw[w] = reinterpret_cast<const float *>(base_ptr + w * kDecodeStages * STAGE_BYTES)[8 * D + h];
+            mstar = fmaxf(mstar, mw[w]);
+        }
+        float acc = 0.f, lsum = 0.f;
+        if (mstar > -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < kDecodeWarps; ++w) {
+                const float *src = reinterpret_cast<const float *>(base_ptr + w * kDecodeStages * STAGE_BYTES);
+                const float wgt = (mw[w] > -INFINITY) ? fast_exp2(mw[w] - mstar) : 0.f;
+                acc += wgt * src[h * D + x];
+                lsum += wgt * src[8 * D + 8 + h];
+            }
+        }
+        const size_t slot = ((size_t)b * p.num_q_heads + (size_t)g * p.group + h) * p.nsplit + split;
+        p.part_o[slot * D + x] = acc;
+        if (x == 0) p.part_ml[slot] = make_float2(mstar, lsum);
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeParams p) {
+    const int bh = blockIdx.x;
+    const int b = bh / p.num_q_heads;
+    const int x = threadIdx.x;
+    int L = p.seq_lens[b];
+    L = max(0, min(L, p.max_blocks * 16));
+    const int ns = (L + p.chunk_tokens - 1) / p.chunk_tokens;
+    const float2 *ml = p.part_ml + (size_t)bh * p.nsplit;
+    const float *po = p.part_o + (size_t)bh * p.nsplit * D;
+    float mstar = -INFINITY;
+    for (int s = 0; s < ns; ++s) mstar = fmaxf(mstar, ml[s].x);
+    float acc = 0.f, lsum = 0.f;
+    if (mstar > -INFINITY) {
+        for (int s = 0; s < ns; ++s) {
+            const float2 v = ml[s];
+            const float w = (v.x > -INFINITY) ? fast_exp2(v.x - mstar) : 0.f;
+            lsum += w * v.y;
+            acc += w * po[(size_t)s * D + x];
+        }
+    }
+    p.out[(size_t)bh * D + x] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
+}
+
+static int chunk_max_tokens() {
+    static int v = [] {
+        int x = 1024;
+        if (const char *e = getenv("EKV_DECODE_CHUNK_MAX")) x = atoi(e);
+        x = (x / 64) * 64;
+        return x < 64 ? 64 : (x > kChunkMaxLimit ? kChunkMaxLimit : x);
+    }();
+    return v;
+}
+
+DecodePlan plan_decode(const ekv_pool *pool, int B, int max_blocks_per_seq) {
+    const int max_len = max_blocks_per_seq * pool->desc.block_size;
+    const long long units = (long long)B * pool->desc.num_kv_heads;
+    const long long target = (long long)pool->sm_count * 2 * 4;  // CTAs: 2 per SM resident, ~4 waves
+    long long want = (target + units - 1) / units;
+    if (want < 1) want = 1;
+    long long chunk = (max_len + want - 1) / want;
+    chunk = (chunk + 63) / 64 * 64;
+    const int cmax = chunk_max_tokens();
+    if (chunk > cmax) chunk = cmax;
+    if (chunk < 64) chunk = 64;
+    DecodePlan plan;
+    plan.chunk_tokens = (int)chunk;
+    plan.nsplit = (int)((max_len + chunk - 1) / chunk);
+    if (plan.nsplit < 1) plan.nsplit = 1;
+    return plan;
+}
+
+static size_t decode_workspace_need(const ekv_pool *pool, int B, int nsplit) {
+    const size_t parts = (size_t)B * pool->desc.num_q_heads * nsplit;
+    const size_t ml = (parts * sizeof(float2) + 255) / 256 * 256;
+    return ml + parts * pool->desc.head_dim * sizeof(float);
+}
+
+template <int D>
+static ekv_status_t launch_decode(ekv_pool *pool, int layer, const DecodeParams &p, int B, cudaStream_t stream) {
+    constexpr int STAGE_BYTES = 2 * (D / 64) * kBoxBytes;
+    const int smem = kDecodeWarps * kDecodeStages * STAGE_BYTES + 1024 + kDecodeWarps * kDecodeStages * 8;
+    static bool attr_set[64] = {false};
+    const int dev = pool->desc.device;
+    if (dev >= 64 || !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode: shared-memory attribute");
+        if (dev < 64) attr_set[dev] = true;
+    }
+    dim3 grid(p.nsplit, pool->desc.num_kv_heads, B);
+    decode_split_kernel<D><<<grid, kDecodeWarps * 32, smem, stream>>>(pool->kv_map[layer], p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode: split launch");
+    decode_combine_kernel<D><<<B * pool->desc.num_q_heads, D, 0, stream>>>(p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode: combine launch");
+    return EKV_OK;
+}
+
+}  // namespace ekv
+
+using namespace ekv;
+
+extern "C" size_t ekv_attn_workspace_bytes(const ekv_pool_t *pool, int32_t max_batch, int32_t max_seq_len) {
+    if (!pool || max_batch < 1 || max_seq_len < 1) return 0;
+    const int max_blocks = (max_seq_len + pool->desc.block_size - 1) / pool->desc.block_size;
+    size_t need = 0;
+    for (int B = 1; B <= max_batch; ++B) {
+        const DecodePlan plan = plan_decode(pool, B, max_blocks);
+        const size_t n = decode_workspace_need(pool, B, plan.nsplit);
+        if (n > need) need = n;
+    }
+    return need;
+}
+
+extern "C" ekv_status_t ekv_attn_decode(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
+                                        const int32_t *block_tables, int32_t max_blocks_per_seq, const int32_t *seq_lens,
+                                        int32_t B, float scale, void *workspace, size_t workspace_bytes, void *stream) {
+    ekv_status_t st = check_compute(pool, layer, "ekv_attn_decode");
+    if (st != EKV_OK) return st;
+    if (B < 0 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26) || B > 65535 ||
+        (B > 0 && (!q || !out || !block_tables || !seq_lens)) || ((uintptr_t)q & 15) || ((uintptr_t)out & 15)) {
+        set_error("ekv_attn_decode: bad argument (B=%d, max_blocks_per_seq=%d)", B, max_blocks_per_seq);
+        return EKV_ERR_INVALID;
+    }
+    if (B == 0) return EKV_OK;
+    const DecodePlan plan = plan_decode(pool, B, max_blocks_per_seq);
+    const size_t need = decode_workspace_need(pool, B, plan.nsplit);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) {
+        set_error("ekv_attn_decode: workspace %p of %zu bytes; need %zu bytes, 256-byte aligned", workspace, workspace_bytes,
+                  need);
+        return EKV_ERR_WORKSPACE;
+    }
+    const size_t parts = (size_t)B * pool->desc.num_q_heads * plan.nsplit;
+    DecodeParams p;
+    p.q = (const __nv_bfloat16 *)q;
+    p.block_tables = block_tables;
+    p.seq_lens = seq_lens;
+    p.live = pool->d_live;
+    p.status = pool->d_status;
+    p.part_ml = (float2 *)workspace;
+    p.part_o = (float *)((uint8_t *)workspace + (parts * sizeof(float2) + 255) / 256 * 256);
+    p.out = (__nv_bfloat16 *)out;
+    p.max_blocks = max_blocks_per_seq;
+    p.num_q_heads = pool->desc.num_q_heads;
+    p.num_kv_heads = pool->desc.num_kv_heads;
+    p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
+    p.chunk_tokens = plan.chunk_tokens;
+    p.nsplit = plan.nsplit;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    if (pool->desc.head_dim == 128) return launch_decode<128>(pool, layer, p, B, (cudaStream_t)stream);
+    return launch_decode<64>(pool, layer, p, B, (cudaStream_t)stream);
+}

@@ -1,0 +1,58 @@
+// ekv_attn_prefill_chunk: host entry point.  Validates, sizes the launch from the host copy of
+// cu_q_lens (no device synchronisation) and dispatches the kernel for the pool's head_dim.
+#include <stdlib.h>
+#include <string.h>
+
+#include "ekv_internal.h"
+#include "ekv_prefill_mma.cuh"
+
+using namespace ekv;
+
+extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
+                                               const int32_t *block_tables, int32_t max_blocks_per_seq,
+                                               const int32_t *cu_q_lens, const int32_t *cu_q_lens_host,
+                                               const int32_t *seq_lens, int32_t R, float scale, void *stream) {
+    ekv_status_t st = check_compute(pool, layer, "ekv_attn_prefill_chunk");
+    if (st != EKV_OK) return st;
+    if (R < 0 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26) ||
+        (R > 0 && (!q || !out || !block_tables || !cu_q_lens || !cu_q_lens_host || !seq_lens)) || ((uintptr_t)q & 15) ||
+        ((uintptr_t)out & 15)) {
+        set_error("ekv_attn_prefill_chunk: bad argument (R=%d, max_blocks_per_seq=%d)", R, max_blocks_per_seq);
+        return EKV_ERR_INVALID;
+    }
+    if (R == 0) return EKV_OK;
+    if (cu_q_lens_host[0] != 0) {
+        set_error("ekv_attn_prefill_chunk: cu_q_lens[0] must be 0");
+        return EKV_ERR_INVALID;
+    }
+    long long q_tiles = 0;
+    for (int r = 0; r < R; ++r) {
+        const int c = cu_q_lens_host[r + 1] - cu_q_lens_host[r];
+        if (c < 0) {
+            set_error("ekv_attn_prefill_chunk: cu_q_lens decreases at request %d", r);
+            return EKV_ERR_INVALID;
+        }
+        q_tiles += (c + kPmBM - 1) / kPmBM;
+    }
+    if (q_tiles == 0) return EKV_OK;
+    if (q_tiles > 0x7fffffffLL) {
+        set_error("ekv_attn_prefill_chunk: too many query tiles");
+        return EKV_ERR_INVALID;
+    }
+    PrefillParams p;
+    p.q = (const __nv_bfloat16 *)q;
+    p.out = (__nv_bfloat16 *)out;
+    p.block_tables = block_tables;
+    p.cu_q_lens = cu_q_lens;
+    p.seq_lens = seq_lens;
+    p.live = pool->d_live;
+    p.status = pool->d_status;
+    p.max_blocks = max_blocks_per_seq;
+    p.num_q_heads = pool->desc.num_q_heads;
+    p.num_kv_heads = pool->desc.num_kv_heads;
+    p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
+    p.R = R;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    if (pool->desc.head_dim == 128) return launch_prefill_mma<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
+    return launch_prefill_mma<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
+}

@@ -1,0 +1,61 @@
+// ekv_write_kv: slot-mapped KV write = exact scatter of bf16 bit patterns into the paged pool.
+// HBM-bound copy: every thread moves one 16-byte piece; a token's K (and V) row of one kv-head is
+// head_dim*2 contiguous bytes on both sides, so loads and stores are fully coalesced.
+#include "ekv_internal.h"
+
+namespace ekv {
+
+// pieces per token = 2 (K,V) * Hkv * (head_dim*2/16)
+__global__ void __launch_bounds__(256) write_kv_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ k,
+                                                       const uint4 *__restrict__ v,
+                                                       const long long *__restrict__ slot_mapping, int T, int num_kv_heads,
+                                                       int block_size, int pieces_per_row,
+                                                       const long long *__restrict__ live_ptr, unsigned *status) {
+    const long long live = *live_ptr;
+    const int row_pieces = num_kv_heads * pieces_per_row;  // one token's K (or V) over all heads
+    const long long total = (long long)T * 2 * row_pieces;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int i = (int)(idx / (2 * row_pieces));
+        const int rem = (int)(idx % (2 * row_pieces));
+        const int kv = rem / row_pieces;
+        const int hp = rem % row_pieces;  // head * pieces_per_row + piece
+        const int h = hp / pieces_per_row, c = hp % pieces_per_row;
+        const long long s = slot_mapping[i];
+        if (s < 0) continue;
+        const long long n = s / block_size;
+        const int t = (int)(s % block_size);
+        if (n >= live) {
+            if (rem == 0) atomicOr(status, EKV_DEV_FLAG_OOB);
+            continue;
+        }
+        const uint4 val = (kv ? v : k)[(long long)i * row_pieces + hp];
+        cache[((((n * 2 + kv) * num_kv_heads + h) * block_size + t) * (long long)pieces_per_row) + c] = val;
+    }
+}
+
+}  // namespace ekv
+
+using namespace ekv;
+
+extern "C" ekv_status_t ekv_write_kv(ekv_pool_t *pool, int32_t layer, const void *k, const void *v,
+                                     const int64_t *slot_mapping, int32_t T, void *stream) {
+    ekv_status_t st = check_compute(pool, layer, "ekv_write_kv");
+    if (st != EKV_OK) return st;
+    if (T < 0 || (T > 0 && (!k || !v || !slot_mapping)) || ((uintptr_t)k & 15) || ((uintptr_t)v & 15)) {
+        set_error("ekv_write_kv: bad argument (T=%d, k=%p, v=%p, slot_mapping=%p)", T, k, v, (const void *)slot_mapping);
+        return EKV_ERR_INVALID;
+    }
+    if (T == 0) return EKV_OK;
+    const int pieces_per_row = pool->desc.head_dim * 2 / 16;
+    const long long total = (long long)T * 2 * pool->desc.num_kv_heads * pieces_per_row;
+    long long blocks = (total + 255) / 256;
+    const long long cap = (long long)pool->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    write_kv_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
+        (uint4 *)pool->va[layer], (const uint4 *)k, (const uint4 *)v, (const long long *)slot_mapping, T,
+        pool->desc.num_kv_heads, pool->desc.block_size, pieces_per_row, pool->d_live, pool->d_status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "ekv_write_kv launch");
+    return EKV_OK;
+}

@@ -1,0 +1,410 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Bit-exact for the KV write and pool bytes; max-abs 2e-2 / mean-abs 2e-3 for bf16-in,
+fp32-accumulate attention outputs."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import ekv_inputs as I
+import oracle
+import paper_2608_23658_b200 as ekv
+from helpers import bf16_bits, cache_view, empty_cache, place_sequence
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+DEV = "cuda:0"
+
+
+def check_close(got_bf16: torch.Tensor, want_f64: np.ndarray, what=""):
+    got = got_bf16.detach().float().cpu().numpy().astype(np.float64)
+    assert got.shape == want_f64.shape, (got.shape, want_f64.shape)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    err = np.abs(got - want_f64)
+    assert err.max() <= MAX_ABS, f"{what}: max-abs {err.max():.4g}"
+    assert err.mean() <= MEAN_ABS, f"{what}: mean-abs {err.mean():.4g}"
+
+
+def seq_kv(seed, L, shape):
+    n = L * shape.num_kv_heads * shape.head_dim
+    K = I.normal_bf16(seed, 1, 0, n).view(L, shape.num_kv_heads, shape.head_dim)
+    V = I.normal_bf16(seed, 2, 0, n).view(L, shape.num_kv_heads, shape.head_dim)
+    return K, V
+
+
+def rand_q(seed, rows, shape):
+    return I.normal_bf16(seed, 3, 0, rows * shape.num_q_heads * shape.head_dim).view(
+        rows, shape.num_q_heads, shape.head_dim)
+
+
+def make_pool(shape, base_blocks, elastic_blocks=0, grown=False, layers=1):
+    return ekv.Pool(num_q_heads=shape.num_q_heads, num_kv_heads=shape.num_kv_heads, head_dim=shape.head_dim,
+                    base_blocks=base_blocks, elastic_blocks=elastic_blocks, num_layers=layers, start_grown=grown)
+
+
+class Case:
+    """A set of sequences placed in a pool (through ekv_write_kv) and mirrored on the host."""
+
+    def __init__(self, shape, lengths, pool_blocks, seed, pool=None, elastic_blocks=0, id_lo=0, perm_seed=None,
+                 max_blocks_per_seq=None, fill_bits=0x7FC0):
+        self.shape = shape
+        self.lengths = torch.as_tensor(lengths, dtype=torch.int64)
+        self.own_pool = pool is None
+        self.pool = pool or make_pool(shape, pool_blocks - elastic_blocks, elastic_blocks, grown=elastic_blocks > 0)
+        info = self.pool.info
+        self.live = info.live_blocks
+        usable = self.live - id_lo if pool_blocks is None else pool_blocks
+        self.tables, self.free_ids = I.assign_blocks(seed if perm_seed is None else perm_seed, 4, self.lengths,
+                                                     shape.block_size, usable, id_lo=id_lo,
+                                                     max_blocks_per_seq=max_blocks_per_seq)
+        self.seqs = [seq_kv(seed * 1000 + b, int(L), shape) for b, L in enumerate(self.lengths)]
+        # device: poison every live block with NaN patterns, then scatter through the library
+        view = self.pool.layer_tensor(0)
+        view.view(torch.int16).fill_(np.array(fill_bits, dtype=np.uint16).view(np.int16).item())
+        self.host = empty_cache(self.live, shape, fill=fill_bits)
+        for b, (K, V) in enumerate(self.seqs):
+            L = int(self.lengths[b])
+            if L == 0:
+                continue
+            slots = I.position_slots(self.tables[b], 0, L, shape.block_size)
+            self.pool.write_kv(0, K.to(DEV), V.to(DEV), slots.to(DEV))
+            place_sequence(self.host, shape, self.tables[b], K, V)
+        torch.cuda.synchronize()
+        self.d_tables = self.tables.to(DEV)
+        self.d_lengths = self.lengths.to(torch.int32).to(DEV)
+
+    def close(self):
+        if self.own_pool:
+            self.pool.close()
+
+    def decode(self, q, scale):
+        return self.pool.attn_decode(0, q.to(DEV), self.d_tables, self.d_lengths, scale)
+
+    def oracle_decode(self, q, scale):
+        s = self.shape
+        return oracle.attn_decode(self.host, s.num_q_heads, s.num_kv_heads, s.block_size, s.head_dim, q,
+                                  self.tables, self.lengths, scale)
+
+
+# --------------------------------------------------------------------------- KV write
+
+
+def test_write_kv_is_an_exact_scatter():
+    shape = I.TINY
+    pool = make_pool(shape, 256, 256, grown=True)
+    try:
+        info = pool.info
+        assert info.live_blocks == 512
+        view = pool.layer_tensor(0)
+        view.view(torch.int16).fill_(0x1234)
+        T = 777
+        K, V = seq_kv(5, T, shape)
+        slots = I.permutation(9, 1, 512 * 16)[:T].clone()
+        slots[::50] = -1
+        pool.write_kv(0, K.to(DEV), V.to(DEV), slots.to(DEV))
+        torch.cuda.synchronize()
+        assert pool.poll_status() == ekv.Status.OK
+        host = empty_cache(512, shape, fill=0x1234)
+        assert oracle.write_kv(host, 512, shape.num_kv_heads, 16, shape.head_dim, K, V, slots) == 0
+        got = bf16_bits(view.cpu()).reshape(-1)
+        assert np.array_equal(got, host)
+    finally:
+        pool.close()
+
+
+def test_write_kv_llama_shape_and_live_limit():
+    shape = I.LLAMA8B
+    pool = make_pool(shape, 64, 32, grown=False)  # elastic range exists but is NOT mapped
+    try:
+        info = pool.info
+        assert (info.base_blocks, info.elastic_blocks, info.live_blocks) == (64, 32, 64)
+        view = pool.layer_tensor(0)
+        view.view(torch.int16).fill_(0x0BAD)
+        T = 300
+        K, V = seq_kv(6, T, shape)
+        slots = I.permutation(10, 1, 64 * 16)[:T].clone()
+        slots[7] = 70 * 16 + 3      # a block in the unmapped elastic range: must be skipped, not touched
+        slots[9] = 5000 * 16        # far outside
+        pool.write_kv(0, K.to(DEV), V.to(DEV), slots.to(DEV))
+        torch.cuda.synchronize()
+        assert pool.poll_status() == ekv.Status.ERR_BLOCK_OOB
+        assert pool.poll_status() == ekv.Status.OK  # read-and-clear
+        host = empty_cache(64, shape, fill=0x0BAD)
+        assert oracle.write_kv(host, 64, shape.num_kv_heads, 16, shape.head_dim, K, V, slots) == 2
+        assert np.array_equal(bf16_bits(view.cpu()).reshape(-1), host)
+    finally:
+        pool.close()
+
+
+# --------------------------------------------------------------------------- decode
+
+
+def test_decode_c1_tiny_paged_step():
+    """configs[0]: 4/2 heads, d64, 512 blocks (256 base + 256 elastic, grown), 8 sequences U[1,512]."""
+    cfg = I.C1
+    lengths = I.decode_lengths(cfg)
+    case = Case(cfg.shape, lengths, 512, cfg.seed, elastic_blocks=256)
+    try:
+        assert (case.tables >= 256).any() and ((case.tables >= 0) & (case.tables < 256)).any()
+        q = rand_q(cfg.seed, len(lengths), cfg.shape)
+        scale = 1 / math.sqrt(cfg.shape.head_dim)
+        out = case.decode(q, scale)
+        check_close(out, case.oracle_decode(q, scale), "C1 decode")
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("shape,lengths", [
+    (I.LLAMA8B, [1, 15, 16, 17, 64, 65, 1000, 2049, 3333]),
+    (I.LLAMA70B, [1, 16, 33, 500, 1025, 2500]),
+    (I.Shape(8, 8, 128), [3, 200, 1100]),       # MHA: group of 1
+    (I.Shape(16, 8, 64), [7, 129, 2100]),
+])
+def test_decode_matches_oracle_across_tiles_and_tails(shape, lengths):
+    need = int(I.blocks_for(torch.tensor(lengths), 16).sum())
+    case = Case(shape, lengths, need + 37, 21)
+    try:
+        q = rand_q(22, len(lengths), shape)
+        scale = 1 / math.sqrt(shape.head_dim)
+        out = case.decode(q, scale)
+        check_close(out, case.oracle_decode(q, scale), f"decode {shape}")
+        again = case.decode(q, scale)
+        assert torch.equal(out, again), "decode is not bitwise reproducible"
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
+
+
+def test_decode_closed_forms_and_empty_sequence():
+    shape = I.LLAMA8B
+    lengths = [1, 0, 40, 1]
+    case = Case(shape, lengths, 16, 31)
+    try:
+        # sequence 2: identical keys -> mean of V
+        K, V = case.seqs[2]
+        K[:] = K[0]
+        slots = I.position_slots(case.tables[2], 0, 40, 16)
+        case.pool.write_kv(0, K.to(DEV), V.to(DEV), slots.to(DEV))
+        q = rand_q(32, 4, shape)
+        out = case.decode(q, 0.09).float().cpu()
+        for b in (0, 3):  # one key: its V row, exactly
+            want = case.seqs[b][1][0].float().repeat_interleave(shape.group, 0)
+            assert torch.equal(out[b], want)
+        assert torch.equal(out[1], torch.zeros_like(out[1]))  # no keys: zeros
+        mean_v = V.double().mean(0).repeat_interleave(shape.group, 0).numpy()
+        assert np.abs(out[2].double().numpy() - mean_v).max() < 4e-3
+    finally:
+        case.close()
+
+
+def test_decode_block_permutation_and_elastic_placement_are_bitwise_invariant():
+    """Same logical data, different physical blocks (all-base, all-elastic, mixed): identical bits."""
+    shape = I.LLAMA8B
+    lengths = [700, 33, 2100, 1]
+    need = int(I.blocks_for(torch.tensor(lengths), 16).sum())
+    pool = make_pool(shape, 256, 256, grown=True)
+    try:
+        info = pool.info
+        q = rand_q(41, len(lengths), shape)
+        outs = []
+        for id_lo, span, perm_seed in [(0, info.base_blocks, 1), (info.base_blocks, info.elastic_blocks, 2),
+                                       (0, info.live_blocks, 3), (0, info.live_blocks, 4)]:
+            assert need <= span
+            case = Case(shape, lengths, span, 40, pool=pool, id_lo=id_lo, perm_seed=perm_seed)
+            outs.append(case.decode(q, 0.088))
+            if id_lo == 0 and span == info.live_blocks:
+                assert (case.tables >= info.base_blocks).any(), "mixed case must straddle the base/elastic line"
+        for o in outs[1:]:
+            assert torch.equal(outs[0], o)
+        check_close(outs[0], case.oracle_decode(q, 0.088), "straddling decode")
+    finally:
+        pool.close()
+
+
+def test_decode_out_of_range_block_id_is_skipped_and_latched():
+    shape = I.LLAMA8B
+    pool = make_pool(shape, 64, 32, grown=False)
+    try:
+        lengths = [100, 50]
+        case = Case(shape, lengths, 64, 51, pool=pool)
+        q = rand_q(52, 2, shape)
+        good = case.decode(q, 0.088)
+        assert pool.poll_status() == ekv.Status.OK
+        bad = case.tables.clone()
+        bad[0, 2] = 80                      # inside the reserved range but NOT live (unmapped)
+        bad[1, 1] = -5
+        out = pool.attn_decode(0, q.to(DEV), bad.to(DEV), case.d_lengths, 0.088)
+        torch.cuda.synchronize()
+        assert pool.poll_status() == ekv.Status.ERR_BLOCK_OOB
+        assert torch.isfinite(out.float()).all()
+        # the skipped block's keys are simply absent: oracle on the shortened key set
+        s = shape
+        K, V = case.seqs[0]
+        keep = torch.cat([torch.arange(0, 32), torch.arange(48, 100)])
+        host = empty_cache(8, s)
+        tbl = torch.arange(8, dtype=torch.int32)[None]
+        place_sequence(host, s, tbl[0], K[keep], V[keep])
+        want = oracle.attn_decode(host, s.num_q_heads, s.num_kv_heads, 16, s.head_dim, q[:1], tbl,
+                                  torch.tensor([len(keep)]), 0.088)
+        check_close(out[:1], want, "decode with a skipped block")
+        assert torch.equal(pool.attn_decode(0, q.to(DEV), case.d_tables, case.d_lengths, 0.088), good)
+    finally:
+        pool.close()
+
+
+def test_decode_argument_errors():
+    shape = I.TINY
+    pool = make_pool(shape, 256)
+    try:
+        q = torch.zeros(2, 4, 64, dtype=torch.bfloat16, device=DEV)
+        bt = torch.zeros(2, 4, dtype=torch.int32, device=DEV)
+        sl = torch.ones(2, dtype=torch.int32, device=DEV)
+        small = torch.empty(256, dtype=torch.uint8, device=DEV)
+        with pytest.raises(ekv.EkvError) as e:
+            pool.attn_decode(0, q, bt, sl, 1.0, workspace=small)
+        assert e.value.status == ekv.Status.ERR_WORKSPACE
+        with pytest.raises(ekv.EkvError) as e:
+            pool.attn_decode(3, q, bt, sl, 1.0)
+        assert e.value.status == ekv.Status.ERR_INVALID
+    finally:
+        pool.close()
+
+
+# --------------------------------------------------------------------------- prefill chunk
+
+
+def run_prefill(case, q, chunks, scale):
+    """chunks: list of (request index, first row of the chunk in the prompt, rows)."""
+    s = case.shape
+    outs = []
+    for (r, start, c) in chunks:
+        cu = torch.tensor([0, c], dtype=torch.int32)
+        out = case.pool.attn_prefill_chunk(0, q[r][start:start + c].contiguous().to(DEV), case.d_tables[r:r + 1].contiguous(),
+                                           cu.to(DEV), cu, torch.tensor([start + c], dtype=torch.int32, device=DEV),
+                                           scale)
+        outs.append(out)
+    return outs
+
+
+def test_prefill_c1_chunk_over_cached_prefix():
+    """configs[0]: one 256-token chunk over a 256-token cached prefix."""
+    cfg = I.C1
+    case = Case(cfg.shape, [512], 512, cfg.seed + 100, elastic_blocks=256)
+    try:
+        s = cfg.shape
+        q = rand_q(cfg.seed + 1, 256, s)
+        scale = 1 / math.sqrt(s.head_dim)
+        (out,) = run_prefill(case, [torch.cat([torch.zeros(256, s.num_q_heads, s.head_dim, dtype=torch.bfloat16), q])],
+                             [(0, 256, 256)], scale)
+        want = oracle.attn_prefill_chunk(case.host, s.num_q_heads, s.num_kv_heads, 16, s.head_dim, q, case.tables,
+                                         np.array([0, 256]), np.array([512]), scale)
+        check_close(out, want, "C1 prefill chunk")
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY, I.LLAMA70B])
+def test_prefill_batched_ragged_requests_match_oracle(shape):
+    chunks = [(0, 1), (0, 100), (37, 64), (500, 129), (130, 300), (1000, 17)]  # (prefix, rows)
+    lengths = [p + c for p, c in chunks]
+    need = int(I.blocks_for(torch.tensor(lengths), 16).sum())
+    case = Case(shape, lengths, need + 11, 61)
+    try:
+        cu = torch.tensor(np.cumsum([0] + [c for _, c in chunks]), dtype=torch.int32)
+        T = int(cu[-1])
+        q = rand_q(62, T, shape)
+        scale = 1 / math.sqrt(shape.head_dim)
+        out = case.pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, case.d_lengths, scale)
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q,
+                                         case.tables, cu, case.lengths, scale)
+        check_close(out, want, f"batched prefill {shape}")
+        assert torch.equal(out, case.pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu,
+                                                             case.d_lengths, scale))
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
+
+
+def test_prefill_chunked_equals_one_shot_and_decode_equals_last_row():
+    shape = I.LLAMA8B
+    L = 1500
+    case = Case(shape, [L], 120, 71)
+    try:
+        q = rand_q(72, L, shape)
+        scale = 1 / math.sqrt(shape.head_dim)
+        (one,) = run_prefill(case, [q], [(0, 0, L)], scale)
+        parts = run_prefill(case, [q], [(0, 0, 1), (0, 1, 500), (0, 501, 487), (0, 988, 512)], scale)
+        chunked = torch.cat(parts)
+        d = (one.float() - chunked.float()).abs()
+        assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q,
+                                         case.tables, np.array([0, L]), np.array([L]), scale)
+        check_close(one, want, "one-shot prefill")
+        check_close(chunked, want, "chunked prefill")
+        dec = case.pool.attn_decode(0, q[-1:].to(DEV), case.d_tables, case.d_lengths, scale)
+        check_close(dec, want[-1:], "decode vs last prefill row")
+    finally:
+        case.close()
+
+
+# --------------------------------------------------------------------------- elastic range
+
+
+def test_elastic_toggle_bytes_pointer_and_outputs():
+    """Outputs for base-resident blocks are bit-identical across shrink/grow; with kept physical
+    memory the elastic bytes read back exactly; the layer pointer never moves."""
+    shape = I.LLAMA8B
+    pool = make_pool(shape, 128, 1024, grown=True, layers=2)
+    try:
+        info = pool.info
+        base, el = info.base_blocks, info.elastic_blocks
+        ptrs = [pool.layer_ptr(l) for l in range(2)]
+        lengths = [900, 77]
+        case = Case(shape, lengths, base, 81, pool=pool)          # tenants of the base range only
+        q = rand_q(82, 2, shape)
+        ref = case.decode(q, 0.088)
+        # seeded bytes into the elastic blocks of both layers
+        for l in range(2):
+            I.fill_normal_bf16_(pool.layer_tensor(l, base, el), 83, 10 + l)
+        before = [pool.layer_tensor(l, base, el).cpu() for l in range(2)]
+
+        ms = pool.shrink(keep_physical=True)
+        assert ms[0] >= 0 and ms[1] >= ms[0]
+        assert not pool.info.grown and pool.info.physical_held and pool.info.live_blocks == base
+        assert torch.equal(case.decode(q, 0.088), ref)
+        pool.grow()
+        assert [pool.layer_ptr(l) for l in range(2)] == ptrs
+        for l in range(2):
+            assert torch.equal(pool.layer_tensor(l, base, el).cpu(), before[l])   # bytes survived the unmap
+        assert torch.equal(case.decode(q, 0.088), ref)
+
+        torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info()[0]
+        pool.shrink()                                               # releasing shrink: memory returns
+        free1 = torch.cuda.mem_get_info()[0]
+        assert not pool.info.physical_held
+        assert free1 - free0 >= 2 * info.elastic_bytes * 0.9
+        assert torch.equal(case.decode(q, 0.088), ref)
+        with pytest.raises(ValueError):
+            pool.layer_tensor(0, base, el)                          # the wrapper refuses unmapped views
+        free2 = torch.cuda.mem_get_info()[0]
+        pool.grow()
+        assert torch.cuda.mem_get_info()[0] <= free2 - 2 * info.elastic_bytes * 0.9
+        # re-granted blocks read back exactly what is written after the remap, K through a copy and
+        # V through the kernel (a one-key sequence returns its V row exactly)
+        K, V = seq_kv(84, 1, shape)
+        blk = base + 5
+        pool.write_kv(1, K.to(DEV), V.to(DEV), torch.tensor([blk * 16], device=DEV))
+        got = pool.layer_tensor(1, blk, 1).cpu()
+        assert torch.equal(got[0, 0, :, 0, :], K[0]) and torch.equal(got[0, 1, :, 0, :], V[0])
+        out = pool.attn_decode(1, q[:1].to(DEV), torch.tensor([[blk]], dtype=torch.int32, device=DEV),
+                               torch.tensor([1], dtype=torch.int32, device=DEV), 0.088)
+        assert torch.equal(out[0].cpu(), V[0].repeat_interleave(shape.group, 0))
+        assert torch.equal(case.decode(q, 0.088), ref)
+        assert pool.poll_status() == ekv.Status.OK
+    finally:
+        pool.close()
