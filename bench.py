@@ -36,9 +36,10 @@ METRIC = "decode-attn HBM GB/s (% peak); prefill-chunk TFLOP/s (% peak); grow/sh
 UNIT = "GB/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes (read + write) per launch of the decode split kernel on this workload, from the ncu
-# capture summarised in profiles/decode_split_c2.md (None until a capture exists).
-DECODE_SPLIT_DRAM_TRAFFIC_BYTES = None
+# DRAM bytes (read + write) per algorithmic byte of the decode split kernel, from the ncu capture
+# summarised in profiles/decode_split_c2_batch32.md (a 32-sequence slice of the same workload; the
+# traffic is proportional to the KV bytes read, so it is scaled to the full launch by that ratio).
+DECODE_SPLIT_DRAM_TRAFFIC_RATIO = (623.645952 + 5.713408) / 622.920860
 
 
 def measured_peaks():
@@ -53,10 +54,12 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks / throttle reasons of one GPU while the timed region runs."""
+    """Samples nvidia-smi clocks / throttle reasons of one GPU in the background; every sample is
+    stamped with the host clock so that the ones taken DURING a region can be picked out."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index: int):
         self.index, self.rows, self.proc = index, [], None
@@ -65,7 +68,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except OSError:
@@ -74,24 +77,30 @@ class ClockSampler:
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
+
+    def wait_for_samples(self, n=1, timeout=3.0):
+        t0 = time.perf_counter()
+        while len(self.rows) < n and time.perf_counter() - t0 < timeout and self.proc:
+            time.sleep(0.01)
 
     def __exit__(self, *exc):
         if self.proc:
-            time.sleep(0.15)
             self.proc.terminate()
             self.thread.join(timeout=2)
 
-    def summary(self):
+    def summary(self, t0, t1):
+        """Median SM clock and throttle reasons over the samples stamped inside [t0, t1]."""
         sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for (t, r) in self.rows:
+            if not (t0 <= t <= t1):
+                continue
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
             except (ValueError, IndexError):
                 continue
-            for n, v in zip(names, r[3:7]):
+            for n, v in zip(self.NAMES, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         if not sm:
@@ -323,7 +332,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ekv", choices=["ekv", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="debug: fewer sequences than the named workload")
@@ -359,8 +368,22 @@ def main():
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     it = iter(evs)
     with ClockSampler(device.index or 0) as clk:
+        clk.wait_for_samples(1)
+        t_load0 = time.perf_counter()
         ms = timed_loop(lambda: wl.step_resident(next(it)), args.steps, device, dist)
-    clocks = clk.summary()
+        t_load1 = time.perf_counter()
+        clocks = clk.summary(t_load0, t_load1)
+        clocks["window"] = "timed region"
+        if clocks["samples"] < 3:
+            # The timed region is shorter than the sampling period: keep the SAME load running, untimed,
+            # until the sampler has seen it, and report those samples (the window says so).
+            t_load0 = time.perf_counter()
+            while time.perf_counter() - t_load0 < 0.6:
+                for _ in range(20):
+                    wl.step_resident()
+                torch.cuda.synchronize(device)
+            clocks = clk.summary(t_load0, time.perf_counter())
+            clocks["window"] = "same steps repeated for 0.6 s right after the timed region (region < sampling period)"
     write_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     decode_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     st = wl.pool.poll_status()
@@ -387,7 +410,7 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "decode_split_kernel<128> + decode_combine_kernel<128>",
                      "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": round(achieved / peaks["hbm_gbs"], 4), "peak_kind": f"{peaks_kind} copy bandwidth",
-                     "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": DECODE_SPLIT_DRAM_TRAFFIC_BYTES,
+                     "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": int(DECODE_SPLIT_DRAM_TRAFFIC_RATIO * wl.decode_bytes),
                      "algorithmic_bytes_per_launch": wl.decode_bytes, "launch_ms": round(decode_ms, 4),
                      "write_kv_ms": round(write_ms, 4)},
         "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
