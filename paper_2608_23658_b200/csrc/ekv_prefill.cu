@@ -5,6 +5,7 @@
 
 #include "ekv_internal.h"
 #include "ekv_prefill_mma.cuh"
+#include "ekv_prefill_tc.cuh"
 
 using namespace ekv;
 
@@ -25,6 +26,16 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
         set_error("ekv_attn_prefill_chunk: cu_q_lens[0] must be 0");
         return EKV_ERR_INVALID;
     }
+    // tcgen05 kernel: head_dim 128, query heads paired inside a kv group, positive scale.  Everything
+    // else (and EKV_PREFILL_IMPL=mma, used by the tests to cross-check the two kernels) takes the
+    // warp-level MMA kernel.
+    static const bool force_mma = [] {
+        const char *e = getenv("EKV_PREFILL_IMPL");
+        return e && strcmp(e, "mma") == 0;
+    }();
+    const int group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
+    const bool use_tc = !force_mma && pool->desc.head_dim == 128 && group % 2 == 0 && scale > 0.f;
+    const int bm = use_tc ? tc::kBM : kPmBM;
     long long q_tiles = 0;
     for (int r = 0; r < R; ++r) {
         const int c = cu_q_lens_host[r + 1] - cu_q_lens_host[r];
@@ -32,7 +43,7 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
             set_error("ekv_attn_prefill_chunk: cu_q_lens decreases at request %d", r);
             return EKV_ERR_INVALID;
         }
-        q_tiles += (c + kPmBM - 1) / kPmBM;
+        q_tiles += (c + bm - 1) / bm;
     }
     if (q_tiles == 0) return EKV_OK;
     if (q_tiles > 0x7fffffffLL) {
@@ -53,6 +64,7 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     p.R = R;
     p.scale_log2 = scale * 1.4426950408889634f;
+    if (use_tc) return tc::launch_prefill_tc(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
     if (pool->desc.head_dim == 128) return launch_prefill_mma<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
     return launch_prefill_mma<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
 }
