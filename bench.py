@@ -203,12 +203,12 @@ def timed_loop(fn, steps, device, dist):
 # ----------------------------------------------------------------------------- side measurements
 
 
-def measure_prefill(device, peaks, reps=3):
+def measure_prefill(device, peaks, reps=3, prompt_len=None, chunks=None):
     """Prefill-chunk TFLOP/s on the configs[2] prompt: 32768 tokens as four 8192-token chunks over
     cached prefixes 0/8k/16k/24k, and as one 32768-token chunk."""
     import paper_2608_23658_b200 as ekv
     cfg, s = I.C3, I.C3.shape
-    Lp = cfg.prompt_len
+    Lp = prompt_len or cfg.prompt_len
     nblk = Lp // s.block_size
     pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=nblk + 64,
                     device=device.index or 0)
@@ -221,7 +221,7 @@ def measure_prefill(device, peaks, reps=3):
         d_table = table.to(device)
         scale = 1.0 / math.sqrt(s.head_dim)
         res = {}
-        for chunk in cfg.chunk_lens:
+        for chunk in (chunks or cfg.chunk_lens):
             calls = []
             for start in range(0, Lp, chunk):
                 cu = torch.tensor([0, chunk], dtype=torch.int32)
@@ -337,6 +337,9 @@ def main():
     ap.add_argument("--impl", default="ekv", choices=["ekv", "reference"])
     ap.add_argument("--batch", type=int, default=None, help="debug: fewer sequences than the named workload")
     ap.add_argument("--no-extras", action="store_true", help="skip prefill / toggle / cpu_baseline side measurements")
+    ap.add_argument("--prefill-only", type=int, default=0, metavar="PROMPT_LEN",
+                    help="profiling aid: run only the prefill-chunk measurement on a prompt of this length "
+                         "(one-shot and in 4 chunks) and print its JSON")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -358,6 +361,10 @@ def main():
         dist = dist_mod
 
     peaks, peaks_kind = measured_peaks()
+    if args.prefill_only:
+        n = args.prefill_only
+        print(json.dumps({"prefill": measure_prefill(device, peaks, reps=2, prompt_len=n, chunks=(n // 4, n))}), flush=True)
+        return
     cfg = I.C2
     wl = DecodeWorkload(cfg, device, args.batch)
     assert wl.decode_bytes > 200e6 or args.batch, "working set must exceed L2"

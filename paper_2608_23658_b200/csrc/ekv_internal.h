@@ -27,7 +27,7 @@ struct ekv_pool {
     std::vector<char> elastic_held;        // per layer: the elastic handle exists
 
     // device state (absent when host_only)
-    long long *d_live;      // device word: number of block ids kernels may dereference
+    long long *d_live;      // device words: [0] number of block ids kernels may dereference, [1] abort word
     unsigned *h_status;     // pinned, host-mapped status word
     unsigned *d_status;     // its device alias
     std::vector<CUtensorMap> kv_map;  // per layer: 2-D view [rows of head_dim bf16], box 64 x block_size, 128B swizzle

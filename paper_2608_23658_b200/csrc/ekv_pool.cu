@@ -377,7 +377,8 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
     }
 
     if (st == EKV_OK && !p->host_only) {
-        cudaError_t e = cudaMalloc((void **)&p->d_live, sizeof(long long));
+        cudaError_t e = cudaMalloc((void **)&p->d_live, 2 * sizeof(long long));  // [0] live limit, [1] abort word
+        if (e == cudaSuccess) e = cudaMemset(p->d_live, 0, 2 * sizeof(long long));
         if (e == cudaSuccess) e = cudaHostAlloc((void **)&p->h_status, sizeof(unsigned), cudaHostAllocMapped);
         if (e == cudaSuccess) {
             *p->h_status = 0;

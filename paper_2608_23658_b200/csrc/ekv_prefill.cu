@@ -1,5 +1,6 @@
 // ekv_attn_prefill_chunk: host entry point.  Validates, sizes the launch from the host copy of
 // cu_q_lens (no device synchronisation) and dispatches the kernel for the pool's head_dim.
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -58,12 +59,35 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     p.seq_lens = seq_lens;
     p.live = pool->d_live;
     p.status = pool->d_status;
+    p.abort_word = reinterpret_cast<int *>(pool->d_live + 1);
     p.max_blocks = max_blocks_per_seq;
     p.num_q_heads = pool->desc.num_q_heads;
     p.num_kv_heads = pool->desc.num_kv_heads;
     p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     p.R = R;
     p.scale_log2 = scale * 1.4426950408889634f;
+    p.trace = nullptr;
+#ifdef EKV_TC_TRACE
+    static unsigned long long *trace_buf = nullptr;
+    if (!trace_buf) cudaMalloc(&trace_buf, 8 * (1 + 2 * 4096));
+    cudaMemsetAsync(trace_buf, 0, 8 * (1 + 2 * 4096), (cudaStream_t)stream);
+    p.trace = trace_buf;
+#endif
+#ifdef EKV_TC_TRACE
+    if (use_tc) {
+        ekv_status_t r = tc::launch_prefill_tc(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
+        cudaStreamSynchronize((cudaStream_t)stream);
+        static unsigned long long host[1 + 2 * 4096];
+        cudaMemcpy(host, p.trace, sizeof host, cudaMemcpyDeviceToHost);
+        unsigned long long n = host[0] > 4096 ? 4096 : host[0], t0 = ~0ull;
+        for (unsigned long long i = 0; i < n; ++i) t0 = host[2 + 2 * i] < t0 ? host[2 + 2 * i] : t0;
+        if (getenv("EKV_TC_TRACE_PRINT"))
+            for (unsigned long long i = 0; i < n; ++i)
+                fprintf(stderr, "trace warp %llu ev %llu j %llu t %llu\n", (host[1 + 2 * i] >> 16) & 0xff, host[1 + 2 * i] & 0xffff,
+                        host[1 + 2 * i] >> 24, host[2 + 2 * i] - t0);
+        return r;
+    }
+#endif
     if (use_tc) return tc::launch_prefill_tc(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
     if (pool->desc.head_dim == 128) return launch_prefill_mma<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
     return launch_prefill_mma<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);

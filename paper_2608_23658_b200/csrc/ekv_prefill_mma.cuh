@@ -23,8 +23,10 @@ struct PrefillParams {
     const int *seq_lens;
     const long long *live;
     unsigned *status;
+    int *abort_word;  // device word: a CTA of this launch gave up on a wait (tcgen05 kernel)
     int max_blocks, num_q_heads, num_kv_heads, group, R;
     float scale_log2;
+    unsigned long long *trace;  // debug builds only (EKV_TC_TRACE): per-role timestamps of one CTA
 };
 
 static constexpr int kPmBM = 64;      // query rows per CTA

@@ -99,6 +99,22 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
     cp::tcgen05_st_32x32b(taddr, r);
 }
 
+#ifdef EKV_TC_TRACE
+#define EKV_TRACE(ev, j)                                                                                   \
+    do {                                                                                                   \
+        if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0) {                    \
+            unsigned long long i_ = atomicAdd(p.trace, 1ull);                                              \
+            if (i_ < 4096) {                                                                               \
+                p.trace[1 + 2 * i_] = (unsigned long long)(ev) | ((unsigned long long)(threadIdx.x >> 5) << 16) | \
+                                      ((unsigned long long)(j) << 24);                                     \
+                p.trace[2 + 2 * i_] = clock64();                                                           \
+            }                                                                                              \
+        }                                                                                                  \
+    } while (0)
+#else
+#define EKV_TRACE(ev, j) do { } while (0)
+#endif
+
 struct Shared {
     uint32_t base;      // shared-window address of the aligned base
     uint8_t *ptr;       // generic pointer to the same place
@@ -109,7 +125,7 @@ struct Shared {
 };
 
 // Bounded wait that also gives up as soon as another role has flagged an abort.
-__device__ __forceinline__ bool wait_or_abort(const Shared &sh, int bar, uint32_t parity, unsigned *status) {
+__device__ __forceinline__ bool wait_or_abort(const Shared &sh, int bar, uint32_t parity, unsigned *status, int *abort_word) {
     const uint32_t b = sh.bar(bar);
     if (mbar_try_wait(b, parity)) return true;
     const uint64_t t0 = global_timer_ns();
@@ -119,6 +135,7 @@ __device__ __forceinline__ bool wait_or_abort(const Shared &sh, int bar, uint32_
             if (*sh.abort_flag()) return false;
             if (global_timer_ns() - t0 > 2000000000ull) {
                 *sh.abort_flag() = 1;
+                *(volatile int *)abort_word = 1;
                 atomicOr(status, EKV_DEV_FLAG_TIMEOUT);
                 return false;
             }
@@ -128,14 +145,15 @@ __device__ __forceinline__ bool wait_or_abort(const Shared &sh, int bar, uint32_
 
 // Warp-uniform form: every lane polls, all lanes agree on the outcome (the roles use warp-collective
 // instructions afterwards, so a warp must leave its loop as a whole).
-__device__ __forceinline__ bool wait_warp(const Shared &sh, int bar, uint32_t parity, unsigned *status) {
-    return __all_sync(0xffffffffu, wait_or_abort(sh, bar, parity, status));
+__device__ __forceinline__ bool wait_warp(const Shared &sh, int bar, uint32_t parity, unsigned *status, int *abort_word) {
+    return __all_sync(0xffffffffu, wait_or_abort(sh, bar, parity, status, abort_word));
 }
 
 __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_constant__ CUtensorMap kvmap,
                                                                  const PrefillParams p) {
-    // a CTA of an earlier wave already timed out: do not start more work on a broken device state
-    if (*(volatile unsigned *)p.status & EKV_DEV_FLAG_TIMEOUT) return;
+    // a CTA of an earlier wave of this launch already timed out: do not start more work (the flag lives
+    // in device memory and is cleared by the launcher; the host-mapped status word is never polled here)
+    if (*(volatile int *)p.abort_word) return;
 
     // ---- which (request, 128-row tile, head pair)?  Heaviest (latest) tiles first.
     const int tile_idx = gridDim.x - 1 - blockIdx.x;
@@ -203,6 +221,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     __syncthreads();
     fence_after();
     const uint32_t tmem = *sh.tmem_slot();
+    EKV_TRACE(1, 0);
 
     if (warp == 0) {
         // =========================== TMA producer ===========================
@@ -234,17 +253,19 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             const int row_k = (my_id * 2 * p.num_kv_heads + g) * 16;
             const uint32_t dst_off = half * kHalfBytes + blk * 2048;
             // K tile
-            if (j >= kStages && !wait_warp(sh, K_EMPTY + s, par_empty, p.status)) break;
+            if (j >= kStages && !wait_warp(sh, K_EMPTY + s, par_empty, p.status, p.abort_word)) break;
             if (lane == 0) {
                 *sh.bad_mask(s) = (int)bad;
                 mbar_expect_tx(sh.bar(K_FULL + s), kTileBytes);
             }
             __syncwarp();
+            EKV_TRACE(10, j);
             if (lane < 16) tma_load_2d(sh.base + kOffK + s * kTileBytes + dst_off, &kvmap, 64 * half, row_k, sh.bar(K_FULL + s));
             // V tile
-            if (j >= kStages && !wait_warp(sh, V_EMPTY + s, par_empty, p.status)) break;
+            if (j >= kStages && !wait_warp(sh, V_EMPTY + s, par_empty, p.status, p.abort_word)) break;
             if (lane == 0) mbar_expect_tx(sh.bar(V_FULL + s), kTileBytes);
             __syncwarp();
+            EKV_TRACE(11, j);
             if (lane >= 16)
                 tma_load_2d(sh.base + kOffV + s * kTileBytes + dst_off, &kvmap, 64 * half, row_k + p.num_kv_heads * 16,
                             sh.bar(V_FULL + s));
@@ -267,7 +288,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 mma_ts(tmem + col_o(x), tmem + col_s(x) + 8 * k, smem_desc(v_addr + k * 2048, kHalfBytes, 1024), kIdescPV,
                        acc || k > 0);
         };
-        bool ok = wait_warp(sh, Q_READY, 0, p.status) && wait_warp(sh, K_FULL + 0, 0, p.status);
+        bool ok = wait_warp(sh, Q_READY, 0, p.status, p.abort_word) && wait_warp(sh, K_FULL + 0, 0, p.status, p.abort_word);
+        EKV_TRACE(20, 0);
         if (ok) {
             fence_after();
             if (lane == 0) {
@@ -281,10 +303,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const int s = j % kStages, s1 = (j + 1) % kStages;
                 const bool more = j + 1 < n_tiles;
-                ok = wait_warp(sh, V_FULL + s, (uint32_t)((j / kStages) & 1), p.status);
-                if (ok && more) ok = wait_warp(sh, K_FULL + s1, (uint32_t)(((j + 1) / kStages) & 1), p.status);
-                if (ok) ok = wait_warp(sh, P_READY + 0, (uint32_t)(j & 1), p.status);
+                ok = wait_warp(sh, V_FULL + s, (uint32_t)((j / kStages) & 1), p.status, p.abort_word);
+                if (ok && more) ok = wait_warp(sh, K_FULL + s1, (uint32_t)(((j + 1) / kStages) & 1), p.status, p.abort_word);
+                EKV_TRACE(21, j);
+                if (ok) ok = wait_warp(sh, P_READY + 0, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
+                EKV_TRACE(22, j);
                 fence_after();
                 if (lane == 0) {
                     issue_pv(0, s, j > 0);
@@ -292,8 +316,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                     mma_commit(sh.bar(S_READY + 0));
                 }
                 __syncwarp();
-                ok = wait_warp(sh, P_READY + 1, (uint32_t)(j & 1), p.status);
+                EKV_TRACE(23, j);
+                ok = wait_warp(sh, P_READY + 1, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
+                EKV_TRACE(24, j);
                 fence_after();
                 if (lane == 0) {
                     issue_pv(1, s, j > 0);
@@ -310,7 +336,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         // every MMA this thread issued must be finished before TMEM is released
         if (lane == 0) mma_commit(sh.bar(DRAIN));
         __syncwarp();
-        (void)wait_warp(sh, DRAIN, 0, p.status);
+        (void)wait_warp(sh, DRAIN, 0, p.status, p.abort_word);
     } else if (warp >= 4) {
         // =========================== softmax + epilogue ===========================
         const int x = (warp - 4) >> 2;                  // 0 = head A, 1 = head B
@@ -339,9 +365,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j % kStages;
-            ok = wait_warp(sh, S_READY + x, (uint32_t)(j & 1), p.status);
+            EKV_TRACE(30, j);
+            ok = wait_warp(sh, S_READY + x, (uint32_t)(j & 1), p.status, p.abort_word);
             if (!ok) break;
             fence_after();
+            EKV_TRACE(31, j);
             const int key0 = j * kBN;
             const int bad = *sh.bad_mask(s);
             const bool need_mask = (key0 + kBN - 1 > prefix + row0) || bad != 0;
@@ -349,7 +377,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             // (unwritten slots): their V rows must not reach the tensor pipe, because 0 * NaN = NaN
             const bool dirty_v = (key0 + kBN > L) || bad != 0;
             if (dirty_v && x == 0) {
-                ok = wait_warp(sh, V_FULL + s, (uint32_t)((j / kStages) & 1), p.status);
+                ok = wait_warp(sh, V_FULL + s, (uint32_t)((j / kStages) & 1), p.status, p.abort_word);
                 if (!ok) break;
                 uint8_t *vdst = sh.ptr + kOffV + s * kTileBytes;
                 if ((key0 + row >= L) || ((bad >> (row >> 4)) & 1)) {  // thread `row` owns key row `row` of the tile
@@ -378,6 +406,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
 #pragma unroll
                 for (int i = 0; i < 32; ++i) mx = fmaxf(mx, sv[i]);
             }
+            EKV_TRACE(32, j);
             const float m_tile = mx * p.scale_log2;  // scale > 0 on this path
             // ---- lazy rescale: raise the reference max only when it is far behind
             const bool raise = m_tile > m_run + kRescaleThreshold;  // also true for the first finite tile
@@ -424,10 +453,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             cp::tcgen05_wait_st();
             fence_before();
             mbar_arrive(sh.bar(P_READY + x));
+            EKV_TRACE(33, j);
         }
 
         // ---- epilogue: O / l -> bf16 -> global (row-contiguous 256 bytes per thread)
-        if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)(n_tiles & 1), p.status);
+        if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)(n_tiles & 1), p.status, p.abort_word);
         if (ok) {
             fence_after();
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
@@ -462,6 +492,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         }
     }
     __syncthreads();
+    EKV_TRACE(99, 0);
     if (warp == 2) cp::tcgen05_dealloc(cp::cta_group_1, tmem, 512);
 }
 
@@ -474,6 +505,8 @@ static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillPa
         if (dev < 64) attr_set[dev] = true;
     }
     dim3 grid(q_tiles, pool->desc.num_q_heads / 2);
+    cudaError_t e0 = cudaMemsetAsync(p.abort_word, 0, sizeof(int), stream);
+    if (e0 != cudaSuccess) return cuda_fail(e0, "ekv_attn_prefill_chunk: clear abort word");
     prefill_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(pool->kv_map[layer], p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_prefill_chunk: launch");
