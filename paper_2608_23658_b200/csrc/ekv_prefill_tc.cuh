@@ -40,6 +40,12 @@ static constexpr int kTileBytes = 2 * kHalfBytes;       // 32 KiB: a Q, K or V t
 static constexpr int kStages = 2;
 static constexpr int kThreads = 384;
 static constexpr float kRescaleThreshold = 8.f;        // log2 units
+// Register re-partition (setmaxnreg): the CTA owns kLaunchRegs x kThreads registers.  Warps 0-3 drop to
+// kRegsUtil, warps 4-11 rise to kRegsSoftmax.  The raise BLOCKS until the pool has the registers, so
+// the split must fit the CTA's own allocation exactly -- nothing else bounds that wait.
+static constexpr int kLaunchRegs = 168, kRegsUtil = 72, kRegsSoftmax = 216;
+static_assert(128 * kRegsUtil + 256 * kRegsSoftmax <= kLaunchRegs * kThreads, "setmaxnreg split exceeds the CTA's registers");
+static_assert(kLaunchRegs * kThreads <= 65536 && kRegsUtil % 8 == 0 && kRegsSoftmax % 8 == 0, "register split");
 
 // shared-memory map (offsets from the 1024-byte aligned base)
 static constexpr int kOffQ = 0;                                   // Q_A, Q_B
@@ -223,11 +229,18 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     const uint32_t tmem = *sh.tmem_slot();
     EKV_TRACE(1, 0);
 
-    if (warp == 0) {
-        // =========================== TMA producer ===========================
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    if (warp == 0 || warp == 2) {
+        // =========================== TMA producers: warp 0 feeds K tiles, warp 2 feeds V tiles ===========
+        // (a TMA issue costs the issuing warp ~100 cycles, 16 boxes per tile: two warps keep up with the MMAs)
+        const bool is_v = warp == 2;
+        const int FULL = is_v ? V_FULL : K_FULL, EMPTY = is_v ? V_EMPTY : K_EMPTY;
+        const uint32_t tile_base = sh.base + (is_v ? kOffV : kOffK);
+        const int kv_row_off = is_v ? p.num_kv_heads * 16 : 0;
         const long long live = *p.live;
         const int *bt = p.block_tables + (size_t)req * p.max_blocks;
-        auto load_id = [&](int j) {  // lanes 0..7: id of block 8j + lane (or -1 past the end / invalid)
+        auto load_id = [&](int j) {  // lane l: id of block 8j + l%8 (-1 past the end, -2 invalid)
             int id = -1;
             const int bi = 8 * j + (lane & 7);
             if (bi < n_blocks) {
@@ -239,36 +252,28 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         int id_next = load_id(0);
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j % kStages;
-            const uint32_t par_empty = (uint32_t)(((j / kStages) - 1) & 1);
             const int id_raw = id_next;
             if (j + 1 < n_tiles) id_next = load_id(j + 1);
             const unsigned oob = __ballot_sync(0xffffffffu, id_raw == -2) & 0xffu;
-            if (oob && lane == 0) atomicOr(p.status, EKV_DEV_FLAG_OOB);
             // blocks whose smem rows will hold stand-in data: invalid ids and blocks past the last visible key
             const unsigned bad = __ballot_sync(0xffffffffu, id_raw < 0) & 0xffu;
             const int id = id_raw < 0 ? 0 : id_raw;  // masked later; block 0 is always mapped
             // box b of a tile: block b/2, channel half b%2  ->  [half][block][16 rows][128 B]
             const int b = lane & 15, blk = b >> 1, half = b & 1;
             const int my_id = __shfl_sync(0xffffffffu, id, blk);
-            const int row_k = (my_id * 2 * p.num_kv_heads + g) * 16;
-            const uint32_t dst_off = half * kHalfBytes + blk * 2048;
-            // K tile
-            if (j >= kStages && !wait_warp(sh, K_EMPTY + s, par_empty, p.status, p.abort_word)) break;
+            const int row = (my_id * 2 * p.num_kv_heads + g) * 16 + kv_row_off;
+            if (j >= kStages && !wait_warp(sh, EMPTY + s, (uint32_t)(((j / kStages) - 1) & 1), p.status, p.abort_word)) break;
             if (lane == 0) {
-                *sh.bad_mask(s) = (int)bad;
-                mbar_expect_tx(sh.bar(K_FULL + s), kTileBytes);
+                if (!is_v) {
+                    if (oob) atomicOr(p.status, EKV_DEV_FLAG_OOB);
+                    *sh.bad_mask(s) = (int)bad;
+                }
+                mbar_expect_tx(sh.bar(FULL + s), kTileBytes);
             }
             __syncwarp();
-            EKV_TRACE(10, j);
-            if (lane < 16) tma_load_2d(sh.base + kOffK + s * kTileBytes + dst_off, &kvmap, 64 * half, row_k, sh.bar(K_FULL + s));
-            // V tile
-            if (j >= kStages && !wait_warp(sh, V_EMPTY + s, par_empty, p.status, p.abort_word)) break;
-            if (lane == 0) mbar_expect_tx(sh.bar(V_FULL + s), kTileBytes);
-            __syncwarp();
-            EKV_TRACE(11, j);
-            if (lane >= 16)
-                tma_load_2d(sh.base + kOffV + s * kTileBytes + dst_off, &kvmap, 64 * half, row_k + p.num_kv_heads * 16,
-                            sh.bar(V_FULL + s));
+            EKV_TRACE(10 + is_v, j);
+            if (lane < 16)
+                tma_load_2d(tile_base + s * kTileBytes + half * kHalfBytes + blk * 2048, &kvmap, 64 * half, row, sh.bar(FULL + s));
         }
     } else if (warp == 1) {
         // =========================== MMA issuer ===========================
@@ -337,7 +342,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         if (lane == 0) mma_commit(sh.bar(DRAIN));
         __syncwarp();
         (void)wait_warp(sh, DRAIN, 0, p.status, p.abort_word);
-    } else if (warp >= 4) {
+    }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // =========================== softmax + epilogue ===========================
         const int x = (warp - 4) >> 2;                  // 0 = head A, 1 = head B
         const int row = ((warp & 3) << 5) | lane;        // query row in the tile = TMEM lane
@@ -390,22 +397,30 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 fence_proxy_async_smem();
             }
 
-            // ---- pass 1: row maximum of the raw scores
-            float mx = -INFINITY;
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                float sv[32];
-                tmem_ld32(sv, t_s + 32 * cc);
-                if (need_mask) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int kk = 32 * cc + i;
-                        if (key0 + kk > lim || ((bad >> (kk >> 4)) & 1)) sv[i] = -INFINITY;
-                    }
-                }
-#pragma unroll
-                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, sv[i]);
+            // ---- the whole score row into registers (one TMEM read), masked entries become -inf
+            float sv[128];
+            {
+                uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
+                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
+                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
+                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
+                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
+                cp::tcgen05_wait_ld();
             }
+            if (need_mask) {
+#pragma unroll
+                for (int i = 0; i < 128; ++i)
+                    if (key0 + i > lim || ((bad >> (i >> 4)) & 1)) sv[i] = -INFINITY;
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 128; i += 4) {
+                mx0 = fmaxf(mx0, sv[i]);
+                mx1 = fmaxf(mx1, sv[i + 1]);
+                mx2 = fmaxf(mx2, sv[i + 2]);
+                mx3 = fmaxf(mx3, sv[i + 3]);
+            }
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             EKV_TRACE(32, j);
             const float m_tile = mx * p.scale_log2;  // scale > 0 on this path
             // ---- lazy rescale: raise the reference max only when it is far behind
@@ -427,28 +442,27 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 }
             }
             const float m_use = m_run > -INFINITY ? m_run : 0.f;
-            // ---- pass 2: P = exp2(S*scale - m), row sum, bf16 pairs back into the S columns
-            float sum = 0.f;
+            // ---- P = exp2(S*scale - m) (a masked -inf gives 0), row sum, bf16 pairs into the S columns
+            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                float sv[32];
-                tmem_ld32(sv, t_s + 32 * cc);
-                uint32_t pk[16];
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t pk[32];
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float a = fast_exp2(fmaf(sv[i], p.scale_log2, -m_use));
-                    float b2 = fast_exp2(fmaf(sv[i + 1], p.scale_log2, -m_use));
-                    if (need_mask) {
-                        const int kk = 32 * cc + i;
-                        if (key0 + kk > lim || ((bad >> (kk >> 4)) & 1)) a = 0.f;
-                        if (key0 + kk + 1 > lim || ((bad >> ((kk + 1) >> 4)) & 1)) b2 = 0.f;
-                    }
-                    sum += a + b2;
-                    pk[i >> 1] = pack_bf16x2(a, b2);
+                for (int i = 0; i < 64; i += 4) {
+                    const float a0 = fast_exp2(fmaf(sv[64 * hh + i], p.scale_log2, -m_use));
+                    const float a1 = fast_exp2(fmaf(sv[64 * hh + i + 1], p.scale_log2, -m_use));
+                    const float a2 = fast_exp2(fmaf(sv[64 * hh + i + 2], p.scale_log2, -m_use));
+                    const float a3 = fast_exp2(fmaf(sv[64 * hh + i + 3], p.scale_log2, -m_use));
+                    sum0 += a0;
+                    sum1 += a1;
+                    sum2 += a2;
+                    sum3 += a3;
+                    pk[i >> 1] = pack_bf16x2(a0, a1);
+                    pk[(i >> 1) + 1] = pack_bf16x2(a2, a3);
                 }
-                // P of keys 32cc..32cc+31 -> 16 packed columns; S columns below 32(cc+1) are already consumed
-                cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
+                cp::tcgen05_st_32x32b(t_s + 32 * hh, pk);
             }
+            const float sum = (sum0 + sum1) + (sum2 + sum3);
             l_run += sum;
             cp::tcgen05_wait_st();
             fence_before();
