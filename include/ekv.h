@@ -181,6 +181,31 @@ EKV_API ekv_status_t ekv_attn_decode(ekv_pool_t *pool, int32_t layer, const void
                              size_t workspace_bytes, void *stream);
 
 /*
+ * ekv_attn_decode_static_scratch -- the paper has no counterpart to this call; it exists for users of
+ * this library who cannot allocate device memory at the moment they need decode attention: an engine
+ * that has already given all free device memory to the KV pool (so that a fresh allocation would
+ * fail, or would take the very reserve ekv_shrink hands back), a C host without any tensor library
+ * or allocator of its own, or code on a path where entering the CUDA allocator is forbidden.
+ * It computes exactly what ekv_attn_decode computes, with the same arguments minus the workspace:
+ * the split pass's fp32 partials go to a fixed array of EKV_STATIC_SCRATCH_BYTES that is part of
+ * the library image (each GPU that loads the library holds it until the process ends).  The call
+ * itself allocates and frees nothing.
+ *   - A call whose split plan needs more than EKV_STATIC_SCRATCH_BYTES is refused with
+ *     EKV_ERR_WORKSPACE and launches nothing (ekv_last_error() states the need); such shapes must use
+ *     ekv_attn_decode.  ekv_attn_workspace_bytes() gives the need of a shape in advance.
+ *   - The first call on a device looks up the array's device address (one cudaGetSymbolAddress with
+ *     that device current) and remembers it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array and find in it whatever the previous call left.
+ *     Nothing in it has to start at zero (every partial that is read was written by the same call),
+ *     so nothing is cleared.  Two calls whose kernels may overlap on the GPU (different streams
+ *     without an ordering between them) race on it: keep them stream-ordered.
+ */
+#define EKV_STATIC_SCRATCH_BYTES (64u << 20)
+EKV_API ekv_status_t ekv_attn_decode_static_scratch(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
+                                                    const int32_t *block_tables, int32_t max_blocks_per_seq,
+                                                    const int32_t *seq_lens, int32_t B, float scale, void *stream);
+
+/*
  * ekv_attn_prefill_chunk -- causal attention of a prompt chunk over its cached prefix plus itself
  * (chunked prefill: "The Decisive Test", "Why the penalty is small": chunking splits the same
  * work across steps).  Request r owns query rows cu_q_lens[r] .. cu_q_lens[r+1]-1 (c_r rows) and

@@ -93,6 +93,7 @@ def load_library():
         "ekv_write_kv": (i32, [vp, i32, vp, vp, vp, i32, vp]),
         "ekv_attn_workspace_bytes": (sz, [vp, i32, i32]),
         "ekv_attn_decode": (i32, [vp, i32, vp, vp, vp, i32, vp, i32, f32, vp, sz, vp]),
+        "ekv_attn_decode_static_scratch": (i32, [vp, i32, vp, vp, vp, i32, vp, i32, f32, vp]),
         "ekv_attn_prefill_chunk": (i32, [vp, i32, vp, vp, vp, i32, vp, vp, vp, i32, f32, vp]),
         "ekv_poll_status": (i32, [vp]),
         "ekv_status_string": (ctypes.c_char_p, [i32]),
@@ -197,6 +198,19 @@ def ekv_attn_decode(pool: int, layer: int, q, out, block_tables, seq_lens, scale
     _check(load_library().ekv_attn_decode(pool, layer, _dptr(q), _dptr(out), _dptr(block_tables), max_blocks,
                                           _dptr(seq_lens), B, float(scale), _dptr(workspace), ws_bytes,
                                           _stream(stream)))
+
+
+EKV_STATIC_SCRATCH_BYTES = 64 << 20
+
+
+def ekv_attn_decode_static_scratch(pool: int, layer: int, q, out, block_tables, seq_lens, scale: float, stream=None):
+    """Decode attention for callers that cannot allocate: same result as ekv_attn_decode, scratch taken
+    from the library's built-in device array (at most EKV_STATIC_SCRATCH_BYTES; larger shapes are refused)."""
+    B = int(seq_lens.shape[0])
+    max_blocks = int(block_tables.shape[1])
+    _check(load_library().ekv_attn_decode_static_scratch(pool, layer, _dptr(q), _dptr(out), _dptr(block_tables),
+                                                         max_blocks, _dptr(seq_lens), B, float(scale),
+                                                         _stream(stream)))
 
 
 def ekv_attn_prefill_chunk(pool: int, layer: int, q, out, block_tables, cu_q_lens, cu_q_lens_host, seq_lens,

@@ -394,3 +394,85 @@ extern "C" ekv_status_t ekv_attn_decode(ekv_pool_t *pool, int32_t layer, const v
     if (pool->desc.head_dim == 128) return launch_decode<128>(pool, layer, p, B, (cudaStream_t)stream);
     return launch_decode<64>(pool, layer, p, B, (cudaStream_t)stream);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Decode attention for callers that cannot allocate.
+//
+// Some users of this library have no allocator to turn to when they need the split pass's scratch:
+// a serving engine that, once started, has handed every free byte of the device to the KV pool (a
+// cudaMalloc then fails or eats the reserve the elastic range gives back), a plain-C host that
+// links no tensor library, or code running where the CUDA allocator must not be entered (inside a
+// stream capture, from a callback).  For them the scratch lives in the library image itself: a
+// fixed device array that every GPU loading the library carries until the process exits.
+// ------------------------------------------------------------------------------------------------
+namespace ekv {
+
+static __device__ __align__(256) unsigned char g_decode_static_scratch[EKV_STATIC_SCRATCH_BYTES];
+
+// In host code the array's name is only a handle for the runtime, not a device address; the address
+// kernels may use is looked up once per device (with that device current) and cached here.
+static void *g_decode_static_scratch_addr[64] = {nullptr};
+
+static ekv_status_t static_scratch_address(int device, void **addr) {
+    if (device < 0 || device >= 64) {
+        set_error("ekv_attn_decode_static_scratch: device ordinal %d is outside the supported 0..63", device);
+        return EKV_ERR_INVALID;
+    }
+    void *ptr = __atomic_load_n(&g_decode_static_scratch_addr[device], __ATOMIC_ACQUIRE);
+    if (ptr == nullptr) {
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_decode_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode_static_scratch: cudaGetSymbolAddress");
+        if (ptr == nullptr || ((uintptr_t)ptr & 255) != 0) {
+            set_error("ekv_attn_decode_static_scratch: scratch symbol resolved to an unusable address %p", ptr);
+            return EKV_ERR_CUDA;
+        }
+        __atomic_store_n(&g_decode_static_scratch_addr[device], ptr, __ATOMIC_RELEASE);
+    }
+    *addr = ptr;
+    return EKV_OK;
+}
+
+}  // namespace ekv
+
+extern "C" ekv_status_t ekv_attn_decode_static_scratch(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
+                                                       const int32_t *block_tables, int32_t max_blocks_per_seq,
+                                                       const int32_t *seq_lens, int32_t B, float scale, void *stream) {
+    ekv_status_t st = check_compute(pool, layer, "ekv_attn_decode_static_scratch");  // makes the pool's device current
+    if (st != EKV_OK) return st;
+    if (B < 0 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26) || B > 65535 ||
+        (B > 0 && (!q || !out || !block_tables || !seq_lens)) || ((uintptr_t)q & 15) || ((uintptr_t)out & 15)) {
+        set_error("ekv_attn_decode_static_scratch: bad argument (B=%d, max_blocks_per_seq=%d)", B, max_blocks_per_seq);
+        return EKV_ERR_INVALID;
+    }
+    if (B == 0) return EKV_OK;
+    const DecodePlan plan = plan_decode(pool, B, max_blocks_per_seq);
+    const size_t need = decode_workspace_need(pool, B, plan.nsplit);
+    if (need > (size_t)EKV_STATIC_SCRATCH_BYTES) {
+        set_error("ekv_attn_decode_static_scratch: this call needs %zu bytes of scratch but the built-in array holds %zu "
+                  "(B=%d, max_blocks_per_seq=%d); use ekv_attn_decode with a caller-provided workspace",
+                  need, (size_t)EKV_STATIC_SCRATCH_BYTES, B, max_blocks_per_seq);
+        return EKV_ERR_WORKSPACE;
+    }
+    void *scratch = nullptr;
+    st = static_scratch_address(pool->desc.device, &scratch);
+    if (st != EKV_OK) return st;
+    const size_t parts = (size_t)B * pool->desc.num_q_heads * plan.nsplit;
+    DecodeParams p;
+    p.q = (const __nv_bfloat16 *)q;
+    p.block_tables = block_tables;
+    p.seq_lens = seq_lens;
+    p.live = pool->d_live;
+    p.status = pool->d_status;
+    p.part_ml = (float2 *)scratch;
+    p.part_o = (float *)((uint8_t *)scratch + (parts * sizeof(float2) + 255) / 256 * 256);
+    p.out = (__nv_bfloat16 *)out;
+    p.max_blocks = max_blocks_per_seq;
+    p.num_q_heads = pool->desc.num_q_heads;
+    p.num_kv_heads = pool->desc.num_kv_heads;
+    p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
+    p.chunk_tokens = plan.chunk_tokens;
+    p.nsplit = plan.nsplit;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    if (pool->desc.head_dim == 128) return launch_decode<128>(pool, layer, p, B, (cudaStream_t)stream);
+    return launch_decode<64>(pool, layer, p, B, (cudaStream_t)stream);
+}
