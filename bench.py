@@ -179,6 +179,20 @@ class DecodeWorkload:
         self.pool.close()
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Replicas run independently; the job's time is the slowest rank's (all-reduce MAX of a device-timed value)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+def whole_job_gbs(step_bytes: int, steps: int, ms: float, world: int) -> float:
+    """Aggregate throughput of `world` replicas that each moved step_bytes per step."""
+    return world * step_bytes * steps / (ms * 1e-3) / 1e9
+
+
 def timed_loop(fn, steps, device, dist):
     """barrier + sync, K steps between two CUDA events on the current stream, sync + barrier; max over ranks."""
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -191,12 +205,9 @@ def timed_loop(fn, steps, device, dist):
         fn()
     e1.record()
     torch.cuda.synchronize(device)
-    ms = e0.elapsed_time(e1)
+    ms = max_over_ranks(e0.elapsed_time(e1), dist, device)
     if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.barrier()
-        ms = float(t[0])
     return ms
 
 
@@ -402,8 +413,8 @@ def main():
     ms_e2e = timed_loop(wl.step_e2e, args.steps, device, dist)
 
     step_bytes = wl.decode_bytes + wl.write_bytes
-    value = world * step_bytes * args.steps / (ms * 1e-3) / 1e9
-    e2e_value = world * step_bytes * args.steps / (ms_e2e * 1e-3) / 1e9
+    value = whole_job_gbs(step_bytes, args.steps, ms, world)
+    e2e_value = whole_job_gbs(step_bytes, args.steps, ms_e2e, world)
     achieved = wl.decode_bytes / (decode_ms * 1e-3) / 1e9
     h2d, d2h = wl.e2e_bytes()
     line = {

@@ -55,19 +55,27 @@ _SIGMA8 = math.sqrt(8.0 * (65536.0 ** 2 - 1.0) / 12.0)
 _INV_SIGMA8 = float(torch.tensor(1.0 / _SIGMA8, dtype=torch.float32))
 
 
-def normal_bf16(seed: int, stream: int, start: int, count: int, device="cpu") -> torch.Tensor:
-    """bf16 values ~N(0,1) for element indices start .. start+count-1 of (seed, stream).
-
-    Element i depends only on (seed, stream, i); identical bits on every device."""
-    key = _key(seed, stream)
-    idx = torch.arange(start, start + count, dtype=torch.int64, device=device)
-    total = torch.zeros(count, dtype=torch.int64, device=device)
+def _normal_from_idx(key: int, idx: torch.Tensor) -> torch.Tensor:
+    total = torch.zeros_like(idx)
     for half in range(2):
         w = mix64((idx * 2 + half) ^ key)
         for f in range(4):
             total += _lsr(w, 16 * f) & 0xFFFF
     centred = (total - 4 * 65535).to(torch.float32)  # |.| < 2^24: exact
     return (centred * _INV_SIGMA8).to(torch.bfloat16)
+
+
+def normal_bf16(seed: int, stream: int, start: int, count: int, device="cpu") -> torch.Tensor:
+    """bf16 values ~N(0,1) for element indices start .. start+count-1 of (seed, stream).
+
+    Element i depends only on (seed, stream, i); identical bits on every device."""
+    idx = torch.arange(start, start + count, dtype=torch.int64, device=device)
+    return _normal_from_idx(_key(seed, stream), idx)
+
+
+def normal_bf16_at(seed: int, stream: int, idx: torch.Tensor) -> torch.Tensor:
+    """The same values at arbitrary element indices (int64 tensor, any device)."""
+    return _normal_from_idx(_key(seed, stream), idx)
 
 
 def fill_normal_bf16_(dst: torch.Tensor, seed: int, stream: int, start: int = 0,
