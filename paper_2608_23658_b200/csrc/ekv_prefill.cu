@@ -77,14 +77,12 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     if (use_tc) {
         ekv_status_t r = tc::launch_prefill_tc(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
         cudaStreamSynchronize((cudaStream_t)stream);
-        static unsigned long long host[1 + 2 * 4096];
+        static unsigned long long host[12 * 8];
         cudaMemcpy(host, p.trace, sizeof host, cudaMemcpyDeviceToHost);
-        unsigned long long n = host[0] > 4096 ? 4096 : host[0], t0 = ~0ull;
-        for (unsigned long long i = 0; i < n; ++i) t0 = host[2 + 2 * i] < t0 ? host[2 + 2 * i] : t0;
         if (getenv("EKV_TC_TRACE_PRINT"))
-            for (unsigned long long i = 0; i < n; ++i)
-                fprintf(stderr, "trace warp %llu ev %llu j %llu t %llu\n", (host[1 + 2 * i] >> 16) & 0xff, host[1 + 2 * i] & 0xffff,
-                        host[1 + 2 * i] >> 24, host[2 + 2 * i] - t0);
+            for (int w = 0; w < 12; ++w)
+                fprintf(stderr, "trace warp %2d: %9llu %9llu %9llu %9llu %9llu %9llu %9llu %9llu\n", w, host[w * 8], host[w * 8 + 1],
+                        host[w * 8 + 2], host[w * 8 + 3], host[w * 8 + 4], host[w * 8 + 5], host[w * 8 + 6], host[w * 8 + 7]);
         return r;
     }
 #endif

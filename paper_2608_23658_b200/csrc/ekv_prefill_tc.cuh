@@ -55,7 +55,7 @@ static constexpr int kOffBar = kOffV + kStages * kTileBytes;      // mbarriers
 static constexpr int kSmemBytes = kOffBar + 256 + 1024;           // + alignment slack
 
 // barrier slots (8 bytes each)
-enum Bar { Q_READY = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_READY = 9, P_READY = 11, DRAIN = 13, NBAR = 14 };
+enum Bar { Q_READY = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_READY = 9, P_READY = 11, DRAIN = 13, P_PART = 14, NBAR = 16 };
 
 // TMEM columns
 __device__ __forceinline__ constexpr uint32_t col_s(int x) { return 128u * (uint32_t)x; }
@@ -105,21 +105,54 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
     cp::tcgen05_st_32x32b(taddr, r);
 }
 
+// Debug builds (EKV_TC_TRACE): every warp of CTA (0,0) accumulates cycles per phase in registers and
+// writes the totals once at the end (slot = warp*8 + phase).
 #ifdef EKV_TC_TRACE
-#define EKV_TRACE(ev, j)                                                                                   \
-    do {                                                                                                   \
-        if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0) {                    \
-            unsigned long long i_ = atomicAdd(p.trace, 1ull);                                              \
-            if (i_ < 4096) {                                                                               \
-                p.trace[1 + 2 * i_] = (unsigned long long)(ev) | ((unsigned long long)(threadIdx.x >> 5) << 16) | \
-                                      ((unsigned long long)(j) << 24);                                     \
-                p.trace[2 + 2 * i_] = clock64();                                                           \
-            }                                                                                              \
-        }                                                                                                  \
+#define EKV_TRACE_DECL long long tr_acc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long tr_t_ = clock64();
+#define EKV_TRACE(ev, j)                          \
+    do {                                          \
+        const long long now_ = clock64();         \
+        tr_acc_[(ev) & 7] += now_ - tr_t_;        \
+        tr_t_ = now_;                             \
+    } while (0)
+#define EKV_TRACE_FLUSH                                                                              \
+    do {                                                                                             \
+        if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0)                \
+            for (int i_ = 0; i_ < 8; ++i_) p.trace[(threadIdx.x >> 5) * 8 + i_] = (unsigned long long)tr_acc_[i_]; \
     } while (0)
 #else
+#define EKV_TRACE_DECL
 #define EKV_TRACE(ev, j) do { } while (0)
+#define EKV_TRACE_FLUSH do { } while (0)
 #endif
+
+#ifndef EKV_TC_PART
+#define EKV_TC_PART 6
+#endif
+#ifndef EKV_TC_EMU
+#define EKV_TC_EMU 0
+#endif
+static constexpr int kPartSteps = EKV_TC_PART;  // PV k-steps (16 keys each) covered by the early P_PART arrival (even, 2..6)
+static constexpr bool kEmulateHalf = EKV_TC_EMU != 0;  // evaluate every second pair of exponentials on the FMA pipe
+
+// 2^x for a pair on the FMA pipe: x = n + f with n = round(x), f in [-0.5, 0.5]; cubic minimax of 2^f
+// (max relative error 7.5e-5, far below the bf16 rounding P gets anyway); 2^n goes into the exponent
+// field by an integer add.  Inputs at or below -126 (masked scores arrive as -inf) return ~1e-38.
+__device__ __forceinline__ float2 exp2_fma_pair(float2 x) {
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 magic = make_float2(12582912.f, 12582912.f);  // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
+    const float2 t = __fadd2_rn(x, magic);
+    const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+    float2 q = __ffma2_rn(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.2426111251f, 0.2426111251f));
+    q = __ffma2_rn(q, f, make_float2(0.6932609677f, 0.6932609677f));
+    q = __ffma2_rn(q, f, make_float2(0.9999280572f, 0.9999280572f));
+    float2 r;
+    r.x = __uint_as_float(__float_as_uint(q.x) + (__float_as_uint(t.x) << 23));
+    r.y = __uint_as_float(__float_as_uint(q.y) + (__float_as_uint(t.y) << 23));
+    return r;
+}
 
 struct Shared {
     uint32_t base;      // shared-window address of the aligned base
@@ -127,7 +160,10 @@ struct Shared {
     __device__ __forceinline__ uint32_t bar(int i) const { return base + kOffBar + 8 * i; }
     __device__ __forceinline__ volatile int *abort_flag() const { return (volatile int *)(ptr + kOffBar + 8 * NBAR); }
     __device__ __forceinline__ uint32_t *tmem_slot() const { return (uint32_t *)(ptr + kOffBar + 8 * NBAR + 8); }
-    __device__ __forceinline__ volatile int *bad_mask(int stage) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 16 + 4 * stage); }
+    // Per-tile mask of key blocks whose shared-memory rows hold stand-in data.  Ring of 4: the K producer
+    // may run two tiles ahead of the softmax warps (it only waits for the QK MMAs), so a slot per STAGE
+    // would be overwritten before the softmax of the older tile has read it.
+    __device__ __forceinline__ volatile int *bad_mask(int tile) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 16 + 4 * (tile & 3)); }
 };
 
 // Bounded wait that also gives up as soon as another role has flagged an abort.
@@ -214,6 +250,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         for (int x = 0; x < 2; ++x) {
             mbar_init(sh.bar(S_READY + x), 1);
             mbar_init(sh.bar(P_READY + x), 128);
+            mbar_init(sh.bar(P_PART + x), 128);
         }
         mbar_init(sh.bar(DRAIN), 1);
         *sh.abort_flag() = 0;
@@ -227,7 +264,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     __syncthreads();
     fence_after();
     const uint32_t tmem = *sh.tmem_slot();
-    EKV_TRACE(1, 0);
+    EKV_TRACE_DECL
 
     if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
@@ -266,14 +303,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             if (lane == 0) {
                 if (!is_v) {
                     if (oob) atomicOr(p.status, EKV_DEV_FLAG_OOB);
-                    *sh.bad_mask(s) = (int)bad;
+                    *sh.bad_mask(j) = (int)bad;
                 }
                 mbar_expect_tx(sh.bar(FULL + s), kTileBytes);
             }
             __syncwarp();
-            EKV_TRACE(10 + is_v, j);
+            EKV_TRACE(0, j);
             if (lane < 16)
                 tma_load_2d(tile_base + s * kTileBytes + half * kHalfBytes + blk * 2048, &kvmap, 64 * half, row, sh.bar(FULL + s));
+            EKV_TRACE(1, j);
         }
     } else if (warp == 1) {
         // =========================== MMA issuer ===========================
@@ -286,15 +324,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 mma_ss(tmem + col_s(x), smem_desc(q_addr[x] + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), kIdescQK, k > 0);
             }
         };
-        auto issue_pv = [&](int x, int s, bool acc) {  // O_x (+)= P_x V(s)
+        auto issue_pv = [&](int x, int s, bool acc, int k0, int k1) {  // O_x (+)= P_x[:, 16k0:16k1] V(s)[16k0:16k1, :]
             const uint32_t v_addr = sh.base + kOffV + s * kTileBytes;
 #pragma unroll
-            for (int k = 0; k < kBN / 16; ++k)
+            for (int k = k0; k < k1; ++k)
                 mma_ts(tmem + col_o(x), tmem + col_s(x) + 8 * k, smem_desc(v_addr + k * 2048, kHalfBytes, 1024), kIdescPV,
                        acc || k > 0);
         };
         bool ok = wait_warp(sh, Q_READY, 0, p.status, p.abort_word) && wait_warp(sh, K_FULL + 0, 0, p.status, p.abort_word);
-        EKV_TRACE(20, 0);
+        EKV_TRACE(7, 0);
         if (ok) {
             fence_after();
             if (lane == 0) {
@@ -310,24 +348,34 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 const bool more = j + 1 < n_tiles;
                 ok = wait_warp(sh, V_FULL + s, (uint32_t)((j / kStages) & 1), p.status, p.abort_word);
                 if (ok && more) ok = wait_warp(sh, K_FULL + s1, (uint32_t)(((j + 1) / kStages) & 1), p.status, p.abort_word);
-                EKV_TRACE(21, j);
-                if (ok) ok = wait_warp(sh, P_READY + 0, (uint32_t)(j & 1), p.status, p.abort_word);
+                EKV_TRACE(0, j);
+                if (ok) ok = wait_warp(sh, P_PART + 0, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
-                EKV_TRACE(22, j);
+                fence_after();
+                if (lane == 0) issue_pv(0, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
+                __syncwarp();
+                ok = wait_warp(sh, P_READY + 0, (uint32_t)(j & 1), p.status, p.abort_word);
+                if (!ok) break;
+                EKV_TRACE(1, j);
                 fence_after();
                 if (lane == 0) {
-                    issue_pv(0, s, j > 0);
+                    issue_pv(0, s, true, kPartSteps, kBN / 16);
                     if (more) issue_qk(0, s1);
                     mma_commit(sh.bar(S_READY + 0));
                 }
                 __syncwarp();
-                EKV_TRACE(23, j);
+                EKV_TRACE(2, j);
+                ok = wait_warp(sh, P_PART + 1, (uint32_t)(j & 1), p.status, p.abort_word);
+                if (!ok) break;
+                fence_after();
+                if (lane == 0) issue_pv(1, s, j > 0, 0, kPartSteps);
+                __syncwarp();
                 ok = wait_warp(sh, P_READY + 1, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
-                EKV_TRACE(24, j);
+                EKV_TRACE(3, j);
                 fence_after();
                 if (lane == 0) {
-                    issue_pv(1, s, j > 0);
+                    issue_pv(1, s, true, kPartSteps, kBN / 16);
                     mma_commit(sh.bar(V_EMPTY + s));
                     if (more) {
                         issue_qk(1, s1);
@@ -372,13 +420,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j % kStages;
-            EKV_TRACE(30, j);
+            EKV_TRACE(4, j);
             ok = wait_warp(sh, S_READY + x, (uint32_t)(j & 1), p.status, p.abort_word);
             if (!ok) break;
             fence_after();
-            EKV_TRACE(31, j);
+            EKV_TRACE(0, j);
             const int key0 = j * kBN;
-            const int bad = *sh.bad_mask(s);
+            const int bad = *sh.bad_mask(j);
             const bool need_mask = (key0 + kBN - 1 > prefix + row0) || bad != 0;
             // keys of this tile that lie past the sequence end, or in a skipped block, may hold anything
             // (unwritten slots): their V rows must not reach the tensor pipe, because 0 * NaN = NaN
@@ -421,7 +469,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 mx3 = fmaxf(mx3, sv[i + 3]);
             }
             const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            EKV_TRACE(32, j);
+            EKV_TRACE(1, j);
             const float m_tile = mx * p.scale_log2;  // scale > 0 on this path
             // ---- lazy rescale: raise the reference max only when it is far behind
             const bool raise = m_tile > m_run + kRescaleThreshold;  // also true for the first finite tile
@@ -443,31 +491,37 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             }
             const float m_use = m_run > -INFINITY ? m_run : 0.f;
             // ---- P = exp2(S*scale - m) (a masked -inf gives 0), row sum, bf16 pairs into the S columns
-            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+            // P of the first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
+            // (EKV_TC_EMU=1 evaluates every second pair of exponentials on the FMA pipe instead of the MUFU
+            // pipe; measured slower on B200 under the 1 kW power cap -- 1.10 vs 1.20-1.25 PFLOP/s -- so off.)
+            float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                uint32_t pk[32];
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 64; i += 4) {
-                    const float a0 = fast_exp2(fmaf(sv[64 * hh + i], p.scale_log2, -m_use));
-                    const float a1 = fast_exp2(fmaf(sv[64 * hh + i + 1], p.scale_log2, -m_use));
-                    const float a2 = fast_exp2(fmaf(sv[64 * hh + i + 2], p.scale_log2, -m_use));
-                    const float a3 = fast_exp2(fmaf(sv[64 * hh + i + 3], p.scale_log2, -m_use));
-                    sum0 += a0;
-                    sum1 += a1;
-                    sum2 += a2;
-                    sum3 += a3;
-                    pk[i >> 1] = pack_bf16x2(a0, a1);
-                    pk[(i >> 1) + 1] = pack_bf16x2(a2, a3);
+                for (int i = 0; i < 32; i += 4) {
+                    const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
+                    const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
+                    const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
+                    const float2 pb = kEmulateHalf ? exp2_fma_pair(xb) : make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+                    acc_a = __fadd2_rn(acc_a, pa);
+                    acc_b = __fadd2_rn(acc_b, pb);
+                    pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
+                    pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
                 }
-                cp::tcgen05_st_32x32b(t_s + 32 * hh, pk);
+                cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
+                if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
+                    cp::tcgen05_wait_st();
+                    fence_before();
+                    mbar_arrive(sh.bar(P_PART + x));
+                }
             }
-            const float sum = (sum0 + sum1) + (sum2 + sum3);
-            l_run += sum;
+            l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
             cp::tcgen05_wait_st();
             fence_before();
             mbar_arrive(sh.bar(P_READY + x));
-            EKV_TRACE(33, j);
+            EKV_TRACE(3, j);
         }
 
         // ---- epilogue: O / l -> bf16 -> global (row-contiguous 256 bytes per thread)
@@ -506,7 +560,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         }
     }
     __syncthreads();
-    EKV_TRACE(99, 0);
+    EKV_TRACE(6, 0);
+    EKV_TRACE_FLUSH;
     if (warp == 2) cp::tcgen05_dealloc(cp::cta_group_1, tmem, 512);
 }
 
