@@ -308,8 +308,9 @@ def measure_toggle(device, cycles=5):
     import paper_2608_23658_b200 as ekv
     cfg, s = I.C5, I.C5.shape
     per_layer = cfg.elastic_total_bytes // cfg.num_layers
-    pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=512,
-                    elastic_blocks=per_layer // s.block_bytes, num_layers=cfg.num_layers, device=device.index or 0)
+    el_blocks = per_layer // s.block_bytes
+    pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=el_blocks + 512,
+                    elastic_blocks=el_blocks, num_layers=cfg.num_layers, device=device.index or 0)
     try:
         rows = {"grow_release": [], "shrink_release": [], "grow_keep": [], "shrink_keep": []}
         for _ in range(cycles):
@@ -322,6 +323,18 @@ def measure_toggle(device, cycles=5):
         out = {k: {"driver_ms_median": round(statistics.median(r[0] for r in v), 3),
                    "call_ms_median": round(statistics.median(r[1] for r in v), 3),
                    "call_ms_max": round(max(r[1] for r in v), 3)} for k, v in rows.items()}
+        # drain: move every elastic block of every layer to a base block (what a decommit does before the unmap)
+        src = torch.arange(pool.info.base_blocks, pool.info.base_blocks + el_blocks, dtype=torch.int32, device=device)
+        dst = torch.arange(0, el_blocks, dtype=torch.int32, device=device)
+        ekv.ekv_move_blocks(pool.handle, src, dst)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ekv.ekv_move_blocks(pool.handle, src, dst)
+        e1.record()
+        torch.cuda.synchronize(device)
+        moved = 2 * cfg.num_layers * el_blocks * s.block_bytes
+        out["drain_move_blocks"] = {"ms": round(e0.elapsed_time(e1), 3), "gbs_read_plus_write": round(moved / e0.elapsed_time(e1) / 1e6, 1),
+                                    "blocks": el_blocks * cfg.num_layers}
         out["workload"] = f"{cfg.num_layers} layers x {per_layer >> 20} MiB elastic, {cycles} cycles per mode"
         out["paper_a100_context_ms"] = {"decommit": 3.0, "commit": 30.0, "naive_commit": 180.0}
         return out

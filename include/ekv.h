@@ -223,6 +223,86 @@ EKV_API ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, con
                                     const int32_t *cu_q_lens, const int32_t *cu_q_lens_host,
                                     const int32_t *seq_lens, int32_t R, float scale, void *stream);
 
+/*
+ * ---- Block pool with a gated elastic id range, drain, and the one-step-ahead controller ----------
+ * Paper, section "An Elastic KV Mechanism": "we gate the top elastic block-id range in the block
+ * pool so those blocks are only handed out when the elastic slice is committed" (paragraph "Two
+ * handles, one virtual range"); "The block pool is a pure integer free list" (section "Background
+ * and Motivation"); "The controller commits the elastic slice during decode-only phases and
+ * decommits it at the boundary before a prefill, with hysteresis ...  Committing grows
+ * num_gpu_blocks and admits the top elastic blocks.  Decommitting first drains those blocks, syncs,
+ * and then unmaps" (paragraph "Controller").
+ *
+ * All of this is host-side bookkeeping (no CUDA call) except ekv_move_blocks.  Intended order of a
+ * decommit:  ekv_blockpool_gate_elastic -> ekv_blockpool_drain_plan -> ekv_move_blocks (+ the caller
+ * rewrites its block tables) -> ekv_blockpool_drain_commit -> ekv_shrink.   Of a commit:
+ * ekv_grow -> ekv_blockpool_admit_elastic.
+ */
+typedef struct ekv_blockpool ekv_blockpool_t;   /* opaque */
+typedef struct ekv_controller ekv_controller_t; /* opaque */
+
+typedef struct ekv_blockpool_stats {
+    int64_t base_blocks, elastic_blocks;
+    int64_t free_base, free_elastic;
+    int64_t elastic_in_use;   /* elastic ids currently handed out (what a drain must move) */
+    int64_t num_gpu_blocks;   /* base_blocks, or base_blocks + elastic_blocks while admitted */
+    int32_t admitted;         /* elastic ids may be handed out */
+    int32_t draining;         /* a drain plan is outstanding */
+} ekv_blockpool_stats_t;
+
+/* Ids 0..base_blocks-1 are base blocks, base_blocks..base_blocks+elastic_blocks-1 elastic blocks
+ * (gated until ekv_blockpool_admit_elastic).  out: HOST. */
+EKV_API ekv_status_t ekv_blockpool_create(int64_t base_blocks, int64_t elastic_blocks, ekv_blockpool_t **out);
+EKV_API ekv_status_t ekv_blockpool_destroy(ekv_blockpool_t *bp);
+/* Hands out n ids (HOST array ids_out), all or nothing: EKV_ERR_OOM and nothing allocated if fewer
+ * are available.  Base ids go first (never-freed ones in ascending order, then most recently freed);
+ * elastic ids only while admitted and only once no base id is free. */
+EKV_API ekv_status_t ekv_blockpool_alloc(ekv_blockpool_t *bp, int64_t n, int32_t *ids_out);
+/* Returns ids to the free list.  Any id that is not currently allocated (or appears twice) fails the
+ * whole call with EKV_ERR_INVALID and frees nothing. */
+EKV_API ekv_status_t ekv_blockpool_free(ekv_blockpool_t *bp, const int32_t *ids, int64_t n);
+/* After ekv_grow: elastic ids may be handed out; num_gpu_blocks grows. */
+EKV_API ekv_status_t ekv_blockpool_admit_elastic(ekv_blockpool_t *bp);
+/* Before ekv_shrink: stop handing out elastic ids; *elastic_in_use (HOST, may be NULL) = how many
+ * are still held by requests. */
+EKV_API ekv_status_t ekv_blockpool_gate_elastic(ekv_blockpool_t *bp, int64_t *elastic_in_use);
+/* Drain plan: for every elastic id in use (ascending) a free base id is reserved; pair i says "move
+ * block from_ids[i] to to_ids[i]".  *n_out = number of pairs.  EKV_ERR_OOM (nothing reserved) if the
+ * base range has too few free blocks -- the caller must preempt requests first; EKV_ERR_INVALID if
+ * capacity < *n_out; EKV_ERR_STATE unless gated and no other drain is outstanding.  HOST arrays.
+ * Until ekv_blockpool_drain_commit the ids of the plan (both sides) must not be freed. */
+EKV_API ekv_status_t ekv_blockpool_drain_plan(ekv_blockpool_t *bp, int32_t *from_ids, int32_t *to_ids, int64_t capacity,
+                                              int64_t *n_out);
+/* After the data was moved and the block tables rewritten: the elastic ids of the plan become free. */
+EKV_API ekv_status_t ekv_blockpool_drain_commit(ekv_blockpool_t *bp);
+EKV_API ekv_status_t ekv_blockpool_stats(const ekv_blockpool_t *bp, ekv_blockpool_stats_t *out);
+
+/* Copies whole blocks src_ids[i] -> dst_ids[i] in EVERY layer of the pool (the data movement of a
+ * drain), asynchronously on `stream`.  src_ids, dst_ids: DEVICE int32 [n]; the two sets must be
+ * disjoint.  Ids outside the live range are skipped and latch EKV_ERR_BLOCK_OOB.  Bit-exact copy. */
+EKV_API ekv_status_t ekv_move_blocks(ekv_pool_t *pool, const int32_t *src_ids, const int32_t *dst_ids, int32_t n, void *stream);
+
+typedef struct ekv_controller_desc {
+    int32_t commit_after_decode_steps; /* hysteresis: commit only after this many consecutive steps without a large prefill (>= 1) */
+    int32_t reserve_prefill_tokens;    /* a step with at least this many prefill tokens needs the activation reserve (>= 1) */
+} ekv_controller_desc_t;
+
+typedef enum ekv_action { EKV_ACT_NONE = 0, EKV_ACT_COMMIT = 1, EKV_ACT_DECOMMIT = 2 } ekv_action_t;
+
+typedef struct ekv_controller_stats {
+    int64_t steps, commits, decommits;
+    int32_t committed, decode_streak;
+} ekv_controller_stats_t;
+
+EKV_API ekv_status_t ekv_controller_create(const ekv_controller_desc_t *desc, int32_t initially_committed, ekv_controller_t **out);
+EKV_API ekv_status_t ekv_controller_destroy(ekv_controller_t *ctrl);
+/* Called at the scheduler boundary with what the scheduler already knows about the NEXT step: its
+ * number of prefill tokens (0 = decode-only).  EKV_ACT_DECOMMIT: the next step needs the reserve, give
+ * it back before running it.  EKV_ACT_COMMIT: the hysteresis window of quiet steps has passed, lend the
+ * reserve to the KV pool.  The controller assumes the caller carries the action out. */
+EKV_API ekv_action_t ekv_controller_decide(ekv_controller_t *ctrl, int32_t next_prefill_tokens);
+EKV_API ekv_status_t ekv_controller_stats(const ekv_controller_t *ctrl, ekv_controller_stats_t *out);
+
 /* Non-blocking read-and-clear of the status latched by kernels (EKV_OK, EKV_ERR_BLOCK_OOB or
  * EKV_ERR_TIMEOUT; the latter wins).  Meaningful after the launching stream was synchronised. */
 EKV_API ekv_status_t ekv_poll_status(ekv_pool_t *pool);

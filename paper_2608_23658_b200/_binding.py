@@ -38,6 +38,24 @@ class PoolDesc(ctypes.Structure):
                 ("elastic_blocks", ctypes.c_int64)]
 
 
+class BlockPoolStats(ctypes.Structure):
+    _fields_ = [("base_blocks", ctypes.c_int64), ("elastic_blocks", ctypes.c_int64), ("free_base", ctypes.c_int64),
+                ("free_elastic", ctypes.c_int64), ("elastic_in_use", ctypes.c_int64), ("num_gpu_blocks", ctypes.c_int64),
+                ("admitted", ctypes.c_int32), ("draining", ctypes.c_int32)]
+
+
+class ControllerDesc(ctypes.Structure):
+    _fields_ = [("commit_after_decode_steps", ctypes.c_int32), ("reserve_prefill_tokens", ctypes.c_int32)]
+
+
+class ControllerStats(ctypes.Structure):
+    _fields_ = [("steps", ctypes.c_int64), ("commits", ctypes.c_int64), ("decommits", ctypes.c_int64),
+                ("committed", ctypes.c_int32), ("decode_streak", ctypes.c_int32)]
+
+
+EKV_ACT_NONE, EKV_ACT_COMMIT, EKV_ACT_DECOMMIT = 0, 1, 2
+
+
 class PoolInfo(ctypes.Structure):
     _fields_ = [("granularity", ctypes.c_uint64), ("block_bytes", ctypes.c_uint64), ("base_bytes", ctypes.c_uint64),
                 ("elastic_bytes", ctypes.c_uint64), ("base_blocks", ctypes.c_int64), ("elastic_blocks", ctypes.c_int64),
@@ -96,6 +114,20 @@ def load_library():
         "ekv_attn_decode_static_scratch": (i32, [vp, i32, vp, vp, vp, i32, vp, i32, f32, vp]),
         "ekv_attn_prefill_chunk": (i32, [vp, i32, vp, vp, vp, i32, vp, vp, vp, i32, f32, vp]),
         "ekv_poll_status": (i32, [vp]),
+        "ekv_blockpool_create": (i32, [i64, i64, ctypes.POINTER(vp)]),
+        "ekv_blockpool_destroy": (i32, [vp]),
+        "ekv_blockpool_alloc": (i32, [vp, i64, vp]),
+        "ekv_blockpool_free": (i32, [vp, vp, i64]),
+        "ekv_blockpool_admit_elastic": (i32, [vp]),
+        "ekv_blockpool_gate_elastic": (i32, [vp, ctypes.POINTER(i64)]),
+        "ekv_blockpool_drain_plan": (i32, [vp, vp, vp, i64, ctypes.POINTER(i64)]),
+        "ekv_blockpool_drain_commit": (i32, [vp]),
+        "ekv_blockpool_stats": (i32, [vp, ctypes.POINTER(BlockPoolStats)]),
+        "ekv_move_blocks": (i32, [vp, vp, vp, i32, vp]),
+        "ekv_controller_create": (i32, [ctypes.POINTER(ControllerDesc), i32, ctypes.POINTER(vp)]),
+        "ekv_controller_destroy": (i32, [vp]),
+        "ekv_controller_decide": (i32, [vp, i32]),
+        "ekv_controller_stats": (i32, [vp, ctypes.POINTER(ControllerStats)]),
         "ekv_status_string": (ctypes.c_char_p, [i32]),
         "ekv_last_error": (ctypes.c_char_p, []),
         "ekv_set_vmm_backend": (i32, [ctypes.POINTER(VmmBackend)]),
@@ -225,3 +257,82 @@ def ekv_attn_prefill_chunk(pool: int, layer: int, q, out, block_tables, cu_q_len
 
 def ekv_poll_status(pool: int) -> Status:
     return Status(load_library().ekv_poll_status(pool))
+
+
+# ---------------------------------------------------------------- block pool, drain, controller
+
+
+def ekv_blockpool_create(base_blocks: int, elastic_blocks: int) -> int:
+    out = ctypes.c_void_p()
+    _check(load_library().ekv_blockpool_create(base_blocks, elastic_blocks, ctypes.byref(out)))
+    return out.value
+
+
+def ekv_blockpool_destroy(bp: int):
+    _check(load_library().ekv_blockpool_destroy(bp))
+
+
+def ekv_blockpool_alloc(bp: int, n: int) -> list:
+    ids = (ctypes.c_int32 * max(n, 1))()
+    _check(load_library().ekv_blockpool_alloc(bp, n, ids))
+    return list(ids[:n])
+
+
+def ekv_blockpool_free(bp: int, ids):
+    arr = (ctypes.c_int32 * max(len(ids), 1))(*ids)
+    _check(load_library().ekv_blockpool_free(bp, arr, len(ids)))
+
+
+def ekv_blockpool_admit_elastic(bp: int):
+    _check(load_library().ekv_blockpool_admit_elastic(bp))
+
+
+def ekv_blockpool_gate_elastic(bp: int) -> int:
+    n = ctypes.c_int64(0)
+    _check(load_library().ekv_blockpool_gate_elastic(bp, ctypes.byref(n)))
+    return int(n.value)
+
+
+def ekv_blockpool_drain_plan(bp: int, capacity: int):
+    """Returns (from_ids, to_ids)."""
+    f = (ctypes.c_int32 * max(capacity, 1))()
+    t = (ctypes.c_int32 * max(capacity, 1))()
+    n = ctypes.c_int64(0)
+    _check(load_library().ekv_blockpool_drain_plan(bp, f, t, capacity, ctypes.byref(n)))
+    return list(f[:n.value]), list(t[:n.value])
+
+
+def ekv_blockpool_drain_commit(bp: int):
+    _check(load_library().ekv_blockpool_drain_commit(bp))
+
+
+def ekv_blockpool_stats(bp: int) -> BlockPoolStats:
+    st = BlockPoolStats()
+    _check(load_library().ekv_blockpool_stats(bp, ctypes.byref(st)))
+    return st
+
+
+def ekv_move_blocks(pool: int, src_ids, dst_ids, stream=None):
+    n = int(src_ids.shape[0])
+    _check(load_library().ekv_move_blocks(pool, _dptr(src_ids), _dptr(dst_ids), n, _stream(stream)))
+
+
+def ekv_controller_create(commit_after_decode_steps: int, reserve_prefill_tokens: int, initially_committed: bool = False) -> int:
+    desc = ControllerDesc(commit_after_decode_steps, reserve_prefill_tokens)
+    out = ctypes.c_void_p()
+    _check(load_library().ekv_controller_create(ctypes.byref(desc), int(initially_committed), ctypes.byref(out)))
+    return out.value
+
+
+def ekv_controller_destroy(ctrl: int):
+    _check(load_library().ekv_controller_destroy(ctrl))
+
+
+def ekv_controller_decide(ctrl: int, next_prefill_tokens: int) -> int:
+    return int(load_library().ekv_controller_decide(ctrl, next_prefill_tokens))
+
+
+def ekv_controller_stats(ctrl: int) -> ControllerStats:
+    st = ControllerStats()
+    _check(load_library().ekv_controller_stats(ctrl, ctypes.byref(st)))
+    return st

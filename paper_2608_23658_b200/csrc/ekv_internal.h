@@ -30,6 +30,7 @@ struct ekv_pool {
     long long *d_live;      // device words: [0] number of block ids kernels may dereference, [1] abort word
     unsigned *h_status;     // pinned, host-mapped status word
     unsigned *d_status;     // its device alias
+    unsigned long long *d_layer_base;  // device array: start address of every layer's range
     std::vector<CUtensorMap> kv_map;  // per layer: 2-D view [rows of head_dim bf16], box 64 x block_size, 128B swizzle
     int sm_count;
 };

@@ -192,6 +192,7 @@ static void teardown(ekv_pool *p) {
         p->be.unreserve(p->be.user, p->va[l], layer_bytes);
     }
     if (p->d_live) cudaFree(p->d_live);
+    if (p->d_layer_base) cudaFree(p->d_layer_base);
     if (p->h_status) cudaFreeHost(p->h_status);
 }
 
@@ -322,6 +323,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
     p->d_live = nullptr;
     p->h_status = nullptr;
     p->d_status = nullptr;
+    p->d_layer_base = nullptr;
     p->sm_count = replaced ? 148 : prop.multiProcessorCount;
     p->block_bytes = 2ull * d.num_kv_heads * d.block_size * d.head_dim * 2ull;
 
@@ -388,6 +390,9 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
             long long live = p->base_blocks + (p->grown ? p->elastic_blocks : 0);
             e = cudaMemcpy(p->d_live, &live, sizeof live, cudaMemcpyHostToDevice);
         }
+        if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_layer_base, sizeof(unsigned long long) * d.num_layers);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(p->d_layer_base, p->va.data(), sizeof(unsigned long long) * d.num_layers, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) st = cuda_fail(e, "ekv_pool_create: device state");
         // One tensor map per layer over the WHOLE range (base + elastic).  Encoding reads no memory,
         // and the map never changes when the elastic slice is mapped or unmapped.
