@@ -303,14 +303,15 @@ def measure_prefill(device, peaks, reps=3, prompt_len=None, chunks=None):
         pool.close()
 
 
-def measure_toggle(device, cycles=5):
-    """grow / shrink ms on the configs[4] geometry: 32 layers x 96 MiB elastic (3 GiB reserve)."""
+def _toggle_modes(device, num_layers, per_layer_bytes, cycles):
+    """grow / shrink ms for one geometry, three ways: keep the range and re-create the handle (default), keep
+    range and handle (EKV_KEEP_PHYSICAL), and the naive way -- a fresh range + handle + mapping per toggle."""
     import paper_2608_23658_b200 as ekv
-    cfg, s = I.C5, I.C5.shape
-    per_layer = cfg.elastic_total_bytes // cfg.num_layers
-    el_blocks = per_layer // s.block_bytes
-    pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=el_blocks + 512,
-                    elastic_blocks=el_blocks, num_layers=cfg.num_layers, device=device.index or 0)
+    s = I.C5.shape
+    el_blocks = per_layer_bytes // s.block_bytes
+    geom = dict(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, num_layers=num_layers,
+                device=device.index or 0)
+    pool = ekv.Pool(base_blocks=el_blocks + 512, elastic_blocks=el_blocks, **geom)
     try:
         rows = {"grow_release": [], "shrink_release": [], "grow_keep": [], "shrink_keep": []}
         for _ in range(cycles):
@@ -332,14 +333,36 @@ def measure_toggle(device, cycles=5):
         ekv.ekv_move_blocks(pool.handle, src, dst)
         e1.record()
         torch.cuda.synchronize(device)
-        moved = 2 * cfg.num_layers * el_blocks * s.block_bytes
+        moved = 2 * num_layers * el_blocks * s.block_bytes
         out["drain_move_blocks"] = {"ms": round(e0.elapsed_time(e1), 3), "gbs_read_plus_write": round(moved / e0.elapsed_time(e1) / 1e6, 1),
-                                    "blocks": el_blocks * cfg.num_layers}
-        out["workload"] = f"{cfg.num_layers} layers x {per_layer >> 20} MiB elastic, {cycles} cycles per mode"
-        out["paper_a100_context_ms"] = {"decommit": 3.0, "commit": 30.0, "naive_commit": 180.0}
-        return out
+                                    "blocks": el_blocks * num_layers}
     finally:
         pool.close()
+    # naive: nothing is kept between toggles -- reserve, create, map and grant a new range per layer at every commit
+    naive_c, naive_d = [], []
+    for _ in range(cycles):
+        torch.cuda.synchronize(device)
+        t0 = time.perf_counter()
+        fresh = ekv.Pool(base_blocks=el_blocks, **geom)
+        t1 = time.perf_counter()
+        fresh.close()
+        t2 = time.perf_counter()
+        naive_c.append((t1 - t0) * 1e3)
+        naive_d.append((t2 - t1) * 1e3)
+    out["naive_commit_fresh_range"] = {"call_ms_median": round(statistics.median(naive_c), 3), "call_ms_max": round(max(naive_c), 3)}
+    out["naive_decommit_fresh_range"] = {"call_ms_median": round(statistics.median(naive_d), 3), "call_ms_max": round(max(naive_d), 3)}
+    out["workload"] = f"{num_layers} layers x {per_layer_bytes >> 20} MiB elastic ({num_layers * per_layer_bytes / 2**30:.2f} GiB), {cycles} cycles per mode"
+    return out
+
+
+def measure_toggle(device, cycles=5):
+    """grow / shrink ms on the configs[4] geometry (32 layers x 96 MiB = 3 GiB) and on the paper's own toggle
+    microbenchmark geometry (28 layers, 3.09 GiB in all; its numbers are from another machine: context only)."""
+    cfg = I.C5
+    out = _toggle_modes(device, cfg.num_layers, cfg.elastic_total_bytes // cfg.num_layers, cycles)
+    out["paper_geometry_28_layers"] = _toggle_modes(device, 28, (int(3.09 * 2**30) // 28 // (2 << 20) + 1) * (2 << 20), cycles)
+    out["paper_a100_context_ms"] = {"decommit": 3.0, "commit": 30.0, "naive_commit": 180.0, "live_decommit": 3.8, "live_commit": 23.8}
+    return out
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
