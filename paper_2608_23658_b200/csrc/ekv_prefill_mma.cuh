@@ -163,7 +163,9 @@ __global__ void __launch_bounds__(128, 2) prefill_mma_kernel(const __grid_consta
         const int tok0 = t * kPmBN;
         int bad_blocks = 0;  // read before the id cache may be refilled below
 #pragma unroll
-        for (int j = 0; j < 4; ++j) bad_blocks |= (ids[(t * 4 + j) % kPmIdCache] < 0 && tok0 + 16 * j < kv_end) ? (1 << j) : 0;
+        // invalid ids AND blocks past the last visible key: both were loaded from a stand-in block whose rows may
+        // hold anything, so their scores are masked and their V rows zeroed (0 * NaN must not reach O)
+        for (int j = 0; j < 4; ++j) bad_blocks |= (ids[(t * 4 + j) % kPmIdCache] < 0) ? (1 << j) : 0;
         // all warps are past tile t-1 here, so its stage may be refilled with tile t+1
         if (t + 1 < n_tiles) {
             if (((t + 1) * 4) % kPmIdCache == 0) {

@@ -133,7 +133,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
 #define EKV_TC_EMU 0
 #endif
 static constexpr int kPartSteps = EKV_TC_PART;  // PV k-steps (16 keys each) covered by the early P_PART arrival (even, 2..6)
-static constexpr bool kEmulateHalf = EKV_TC_EMU != 0;  // evaluate every second pair of exponentials on the FMA pipe
+static constexpr int kEmulatePairsOf8 = EKV_TC_EMU;  // of every 8 pairs of exponentials, how many go to the FMA pipe instead of the MUFU pipe
 
 // 2^x for a pair on the FMA pipe: x = n + f with n = round(x), f in [-0.5, 0.5]; cubic minimax of 2^f
 // (max relative error 7.5e-5, far below the bf16 rounding P gets anyway); 2^n goes into the exponent
@@ -504,7 +504,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                     const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
                     const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
                     const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
-                    const float2 pb = kEmulateHalf ? exp2_fma_pair(xb) : make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+                    // pairs are numbered i/2 (MUFU first) and i/2+1; the second one of a group is emulated while the
+                    // group index (i/4 of 8) is below the configured count
+                    const float2 pb = ((i >> 2) < kEmulatePairsOf8) ? exp2_fma_pair(xb) : make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
                     acc_a = __fadd2_rn(acc_a, pa);
                     acc_b = __fadd2_rn(acc_b, pb);
                     pk[i >> 1] = pack_bf16x2(pa.x, pa.y);

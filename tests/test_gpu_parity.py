@@ -408,3 +408,62 @@ def test_elastic_toggle_bytes_pointer_and_outputs():
         assert pool.poll_status() == ekv.Status.OK
     finally:
         pool.close()
+
+
+def test_prefill_edge_cases_bad_ids_empty_requests_and_both_kernels_agree():
+    """Out-of-range block ids inside a prompt are skipped and latched (both prefill kernels); requests with zero
+    rows are legal; the tcgen05 kernel and the warp-MMA kernel agree within tolerance on the same call."""
+    import os
+    import subprocess
+    import sys
+    shape = I.LLAMA8B
+    pool = make_pool(shape, 128, 32, grown=False)
+    try:
+        chunks = [(0, 0), (200, 150), (0, 0), (64, 1)]               # (prefix, rows); two empty requests
+        lengths = [p + c for p, c in chunks]
+        case = Case(shape, lengths, 128, 91, pool=pool)
+        cu = torch.tensor(np.cumsum([0] + [c for _, c in chunks]), dtype=torch.int32)
+        q = rand_q(92, int(cu[-1]), shape)
+        scale = 1 / math.sqrt(shape.head_dim)
+        out = pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, case.d_lengths, scale)
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q, case.tables,
+                                         cu, case.lengths, scale)
+        check_close(out, want, "prefill with empty requests")
+        assert pool.poll_status() == ekv.Status.OK
+        # a block of the prompt points into the unmapped elastic range: its 16 keys are skipped
+        bad = case.tables.clone()
+        bad[1, 3] = 140
+        outb = pool.attn_prefill_chunk(0, q.to(DEV), bad.to(DEV), cu.to(DEV), cu, case.d_lengths, scale)
+        torch.cuda.synchronize()
+        assert pool.poll_status() == ekv.Status.ERR_BLOCK_OOB
+        K, V = case.seqs[1]
+        keep = torch.cat([torch.arange(0, 48), torch.arange(64, 350)])
+        nb = (len(keep) + 15) // 16
+        # oracle with the 16 keys removed: rows keep their causal limits, so restate them as shifted positions
+        host = empty_cache(nb + 1, shape)
+        tbl = torch.arange(nb, dtype=torch.int32)[None]
+        place_sequence(host, shape, tbl[0], K[keep], V[keep])
+        qs = q[int(cu[1]):int(cu[2])]
+        wantb = oracle.attn_prefill_chunk(host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, qs, tbl,
+                                          np.array([0, 150]), np.array([len(keep)]), scale)
+        check_close(outb[int(cu[1]):int(cu[2])], wantb, "prefill with a skipped block")
+        # negative scale takes the warp-MMA kernel; compare with the oracle too
+        outn = pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, case.d_lengths, -scale)
+        wantn = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q,
+                                          case.tables, cu, case.lengths, -scale)
+        check_close(outn, wantn, "prefill with a negative scale")
+        assert pool.poll_status() == ekv.Status.OK
+    finally:
+        pool.close()
+    # the same call through each kernel (selected by the environment when the library is first used): one
+    # process per kernel, see tests/prefill_impl_probe.py
+    import tempfile
+    probe = os.path.join(os.path.dirname(os.path.abspath(__file__)), "prefill_impl_probe.py")
+    with tempfile.TemporaryDirectory() as d:
+        outs = {}
+        for impl in ("mma", "tc"):
+            path = os.path.join(d, impl + ".pt")
+            subprocess.run([sys.executable, probe, path], check=True, env=dict(os.environ, EKV_PREFILL_IMPL=impl))
+            outs[impl] = torch.load(path)
+        diff = (outs["mma"].float() - outs["tc"].float()).abs()
+        assert diff.max().item() <= MAX_ABS and diff.mean().item() <= MEAN_ABS
