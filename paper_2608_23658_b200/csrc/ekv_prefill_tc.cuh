@@ -85,6 +85,39 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)acc)
         : "memory");
 }
+// The single MMA-issuing thread is the pace-setter of the whole CTA, so its instruction count per MMA matters:
+// every shared-memory descriptor used here has the same upper word (stride byte offset 1024, version 1, 128-byte
+// swizzle), and the lower word is (address >> 4) | (leading byte offset >> 4) << 16, so stepping through a tile
+// is one 32-bit add per operand.
+static constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+    return ((addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+template <bool kAcc>
+__device__ __forceinline__ void mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHi), "r"(idesc), "n"(kAcc ? 1 : 0)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ss_lo_dyn(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHi), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_lo_dyn(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHi), "r"(idesc), "r"(acc)
+        : "memory");
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -315,21 +348,23 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         }
     } else if (warp == 1) {
         // =========================== MMA issuer ===========================
-        const uint32_t q_addr[2] = {sh.base + kOffQ, sh.base + kOffQ + kTileBytes};
+        // descriptor low words of the tile origins; stepping inside a tile adds a compile-time constant
+        const uint32_t q_lo[2] = {desc_lo(sh.base + kOffQ, 16), desc_lo(sh.base + kOffQ + kTileBytes, 16)};
+        const uint32_t k_lo0 = desc_lo(sh.base + kOffK, 16), v_lo0 = desc_lo(sh.base + kOffV, kHalfBytes);
         auto issue_qk = [&](int x, int s) {  // S_x = Q_x K(s)^T
-            const uint32_t k_addr = sh.base + kOffK + s * kTileBytes;
+            const uint32_t k_lo = k_lo0 + (uint32_t)s * (kTileBytes >> 4);
 #pragma unroll
             for (int k = 0; k < kD / 16; ++k) {
-                const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-                mma_ss(tmem + col_s(x), smem_desc(q_addr[x] + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), kIdescQK, k > 0);
+                const uint32_t off = ((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4;
+                if (k == 0) mma_ss_lo<false>(tmem + col_s(x), q_lo[x] + off, k_lo + off, kIdescQK);
+                else mma_ss_lo<true>(tmem + col_s(x), q_lo[x] + off, k_lo + off, kIdescQK);
             }
         };
         auto issue_pv = [&](int x, int s, bool acc, int k0, int k1) {  // O_x (+)= P_x[:, 16k0:16k1] V(s)[16k0:16k1, :]
-            const uint32_t v_addr = sh.base + kOffV + s * kTileBytes;
+            const uint32_t v_lo = v_lo0 + (uint32_t)s * (kTileBytes >> 4);
 #pragma unroll
             for (int k = k0; k < k1; ++k)
-                mma_ts(tmem + col_o(x), tmem + col_s(x) + 8 * k, smem_desc(v_addr + k * 2048, kHalfBytes, 1024), kIdescPV,
-                       acc || k > 0);
+                mma_ts_lo_dyn(tmem + col_o(x), tmem + col_s(x) + 8 * k, v_lo + ((k * 2048) >> 4), kIdescPV, (acc || k > 0) ? 1u : 0u);
         };
         bool ok = wait_warp(sh, Q_READY, 0, p.status, p.abort_word) && wait_warp(sh, K_FULL + 0, 0, p.status, p.abort_word);
         EKV_TRACE(7, 0);
