@@ -5,32 +5,50 @@
 
 namespace ekv {
 
-// pieces per token = 2 (K,V) * Hkv * (head_dim*2/16)
-__global__ void __launch_bounds__(256) write_kv_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ k,
-                                                       const uint4 *__restrict__ v,
-                                                       const long long *__restrict__ slot_mapping, int T, int num_kv_heads,
-                                                       int block_size, int pieces_per_row,
-                                                       const long long *__restrict__ live_ptr, unsigned *status) {
+// One token's K and V rows are 2 * Hkv * (head_dim*2/16) pieces of 16 bytes.  A CTA walks over tokens; its
+// threads cover a contiguous chunk of pieces at a time, issuing all loads of the chunk before its stores so
+// that several 16-byte requests per thread are in flight.
+static constexpr int kWriteThreads = 256;
+static constexpr int kWriteUnroll = 4;
+
+__global__ void __launch_bounds__(kWriteThreads) write_kv_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ k,
+                                                                 const uint4 *__restrict__ v,
+                                                                 const long long *__restrict__ slot_mapping, int T,
+                                                                 int num_kv_heads, int block_size, int pieces_per_row,
+                                                                 const long long *__restrict__ live_ptr, unsigned *status) {
     const long long live = *live_ptr;
     const int row_pieces = num_kv_heads * pieces_per_row;  // one token's K (or V) over all heads
-    const long long total = (long long)T * 2 * row_pieces;
-    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * blockDim.x) {
-        const int i = (int)(idx / (2 * row_pieces));
-        const int rem = (int)(idx % (2 * row_pieces));
-        const int kv = rem / row_pieces;
-        const int hp = rem % row_pieces;  // head * pieces_per_row + piece
-        const int h = hp / pieces_per_row, c = hp % pieces_per_row;
-        const long long s = slot_mapping[i];
-        if (s < 0) continue;
-        const long long n = s / block_size;
-        const int t = (int)(s % block_size);
-        if (n >= live) {
-            if (rem == 0) atomicOr(status, EKV_DEV_FLAG_OOB);
-            continue;
+    const int token_pieces = 2 * row_pieces;
+    const long long total = (long long)T * token_pieces;
+    // a CTA takes contiguous chunks of kWriteThreads * kWriteUnroll pieces (16 KiB of source rows)
+    const long long chunk = (long long)kWriteThreads * kWriteUnroll;
+    for (long long base = (long long)blockIdx.x * chunk + threadIdx.x; base < total + threadIdx.x; base += (long long)gridDim.x * chunk) {
+        uint4 val[kWriteUnroll];
+        long long dst[kWriteUnroll];
+#pragma unroll
+        for (int u = 0; u < kWriteUnroll; ++u) {
+            const long long idx = base + (long long)u * kWriteThreads;
+            dst[u] = -1;
+            if (idx >= total) continue;
+            const int i = (int)(idx / token_pieces);
+            const int rem = (int)(idx - (long long)i * token_pieces);
+            const int kv = rem >= row_pieces;
+            const int hp = rem - kv * row_pieces;  // head * pieces_per_row + piece
+            const int h = hp / pieces_per_row, c = hp - h * pieces_per_row;
+            const long long s = slot_mapping[i];
+            if (s < 0) continue;
+            const long long n = s / block_size;
+            const int t = (int)(s - n * block_size);
+            if (n >= live) {
+                if (rem == 0) atomicOr(status, EKV_DEV_FLAG_OOB);
+                continue;
+            }
+            val[u] = (kv ? v : k)[(long long)i * row_pieces + hp];
+            dst[u] = ((((n * 2 + kv) * num_kv_heads + h) * block_size + t) * (long long)pieces_per_row) + c;
         }
-        const uint4 val = (kv ? v : k)[(long long)i * row_pieces + hp];
-        cache[((((n * 2 + kv) * num_kv_heads + h) * block_size + t) * (long long)pieces_per_row) + c] = val;
+#pragma unroll
+        for (int u = 0; u < kWriteUnroll; ++u)
+            if (dst[u] >= 0) cache[dst[u]] = val[u];
     }
 }
 
@@ -49,10 +67,10 @@ extern "C" ekv_status_t ekv_write_kv(ekv_pool_t *pool, int32_t layer, const void
     if (T == 0) return EKV_OK;
     const int pieces_per_row = pool->desc.head_dim * 2 / 16;
     const long long total = (long long)T * 2 * pool->desc.num_kv_heads * pieces_per_row;
-    long long blocks = (total + 255) / 256;
-    const long long cap = (long long)pool->sm_count * 16;
+    long long blocks = (total + kWriteThreads * kWriteUnroll - 1) / (kWriteThreads * kWriteUnroll);
+    const long long cap = (long long)pool->sm_count * 8;  // 8 CTAs of 256 threads per SM: one full wave
     if (blocks > cap) blocks = cap;
-    write_kv_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
+    write_kv_kernel<<<(unsigned)blocks, kWriteThreads, 0, (cudaStream_t)stream>>>(
         (uint4 *)pool->va[layer], (const uint4 *)k, (const uint4 *)v, (const long long *)slot_mapping, T,
         pool->desc.num_kv_heads, pool->desc.block_size, pieces_per_row, pool->d_live, pool->d_status);
     cudaError_t e = cudaGetLastError();
