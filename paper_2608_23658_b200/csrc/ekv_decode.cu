@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeParams p)
 
 static int chunk_max_tokens() {
     static int v = [] {
-        int x = 1024;
+        int x = 2048;
         if (const char *e = getenv("EKV_DECODE_CHUNK_MAX")) x = atoi(e);
         x = (x / 64) * 64;
         return x < 64 ? 64 : (x > kChunkMaxLimit ? kChunkMaxLimit : x);
