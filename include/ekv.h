@@ -206,6 +206,22 @@ EKV_API ekv_status_t ekv_attn_decode_static_scratch(ekv_pool_t *pool, int32_t la
                                                     const int32_t *seq_lens, int32_t B, float scale, void *stream);
 
 /*
+ * ekv_attn_decode_two_tensor -- the alternative the paper weighs and rejects in "The contiguity
+ * constraint": "split the KV into two tensors and rewrite the kernel to read both".  Same computation
+ * and arguments as ekv_attn_decode, except that block ids 0..base_blocks-1 address the pool's base
+ * range of `layer` and ids base_blocks..base_blocks+second_blocks-1 address `second_tensor`, a
+ * separately allocated DEVICE buffer of second_blocks*block_bytes with the same block layout (16-byte
+ * aligned; the pool's elastic range plays no part and may be unmapped).  Ids at or beyond
+ * base_blocks+second_blocks are skipped and latch EKV_ERR_BLOCK_OOB.  It exists to measure what the
+ * single-range design saves (a second tensor map and a choice per block inside the kernel); results
+ * are bitwise identical to ekv_attn_decode on the same logical data.
+ */
+EKV_API ekv_status_t ekv_attn_decode_two_tensor(ekv_pool_t *pool, int32_t layer, const void *second_tensor,
+                                                int64_t second_blocks, const void *q, void *out, const int32_t *block_tables,
+                                                int32_t max_blocks_per_seq, const int32_t *seq_lens, int32_t B, float scale,
+                                                void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * ekv_attn_prefill_chunk -- causal attention of a prompt chunk over its cached prefix plus itself
  * (chunked prefill: "The Decisive Test", "Why the penalty is small": chunking splits the same
  * work across steps).  Request r owns query rows cu_q_lens[r] .. cu_q_lens[r+1]-1 (c_r rows) and

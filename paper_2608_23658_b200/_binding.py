@@ -111,6 +111,7 @@ def load_library():
         "ekv_write_kv": (i32, [vp, i32, vp, vp, vp, i32, vp]),
         "ekv_attn_workspace_bytes": (sz, [vp, i32, i32]),
         "ekv_attn_decode": (i32, [vp, i32, vp, vp, vp, i32, vp, i32, f32, vp, sz, vp]),
+        "ekv_attn_decode_two_tensor": (i32, [vp, i32, vp, i64, vp, vp, vp, i32, vp, i32, f32, vp, sz, vp]),
         "ekv_attn_decode_static_scratch": (i32, [vp, i32, vp, vp, vp, i32, vp, i32, f32, vp]),
         "ekv_attn_prefill_chunk": (i32, [vp, i32, vp, vp, vp, i32, vp, vp, vp, i32, f32, vp]),
         "ekv_poll_status": (i32, [vp]),
@@ -230,6 +231,21 @@ def ekv_attn_decode(pool: int, layer: int, q, out, block_tables, seq_lens, scale
     _check(load_library().ekv_attn_decode(pool, layer, _dptr(q), _dptr(out), _dptr(block_tables), max_blocks,
                                           _dptr(seq_lens), B, float(scale), _dptr(workspace), ws_bytes,
                                           _stream(stream)))
+
+
+def ekv_attn_decode_two_tensor(pool: int, layer: int, second_tensor, q, out, block_tables, seq_lens, scale: float, workspace,
+                               stream=None):
+    """Decode over two tensors: ids below the pool's base_blocks address the pool, the others `second_tensor`
+    (a torch tensor of whole blocks in the pool's block layout)."""
+    B = int(seq_lens.shape[0])
+    max_blocks = int(block_tables.shape[1])
+    info = ekv_pool_info(pool)
+    nbytes = second_tensor.numel() * second_tensor.element_size()
+    assert nbytes % info.block_bytes == 0
+    ws_bytes = workspace.numel() * workspace.element_size()
+    _check(load_library().ekv_attn_decode_two_tensor(pool, layer, _dptr(second_tensor), nbytes // info.block_bytes, _dptr(q),
+                                                     _dptr(out), _dptr(block_tables), max_blocks, _dptr(seq_lens), B,
+                                                     float(scale), _dptr(workspace), ws_bytes, _stream(stream)))
 
 
 EKV_STATIC_SCRATCH_BYTES = 64 << 20

@@ -43,11 +43,16 @@ struct DecodeParams {
     int max_blocks, num_q_heads, num_kv_heads, group;
     int chunk_tokens, nsplit;
     float scale_log2;
+    long long first_tensor_blocks;  // two-tensor variant only: ids below this live in the first tensor
+    long long total_blocks;         // two-tensor variant only: ids at or above this are invalid
 };
 
-template <int D>
+// kTwo = false: the paper's arrangement, one tensor map over the layer's single virtual range.
+// kTwo = true: the alternative the paper rejected (two tensors, the kernel reads both): ids at or above
+// p.first_tensor_blocks address a second, separately allocated tensor through kvmap2.
+template <int D, bool kTwo>
 __global__ void __launch_bounds__(kDecodeWarps * 32, 2)
-decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const DecodeParams p) {
+decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const __grid_constant__ CUtensorMap kvmap2, const DecodeParams p) {
     constexpr int BOXES = D / 64;
     constexpr int TILE_BYTES = BOXES * kBoxBytes;
     constexpr int STAGE_BYTES = 2 * TILE_BYTES;
@@ -75,13 +80,14 @@ decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const DecodeParam
 
     if (lane == 0) {
         prefetch_tensormap(&kvmap);
+        if (kTwo) prefetch_tensormap(&kvmap2);
         for (int s = 0; s < kDecodeStages; ++s) mbar_init(my_bars + 8 * s, 1);
         mbar_fence_init();
     }
     __syncwarp();
 
     // Block ids of this warp's blocks: lane i holds the id of its i-th block.
-    const long long live = *p.live;
+    const long long live = kTwo ? p.total_blocks : *p.live;
     const int *bt = p.block_tables + (size_t)b * p.max_blocks + (t_begin >> 4) + warp;
     int my_id = (lane < nw) ? bt[lane * kDecodeWarps] : 0;
     const bool my_ok = (lane < nw) && my_id >= 0 && (long long)my_id < live;
@@ -90,18 +96,23 @@ decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const DecodeParam
 
     const uint64_t policy = policy_evict_first();
     auto issue = [&](int i) {
-        const int id = __shfl_sync(FULL, my_id, i);
+        int id = __shfl_sync(FULL, my_id, i);
         if (lane == 0 && ((valid_mask >> i) & 1u)) {
             const int stage = i % kDecodeStages;
             const uint32_t bar = my_bars + 8 * stage;
             const uint32_t dst = my_stages + stage * STAGE_BYTES;
+            const CUtensorMap *map = &kvmap;
+            if (kTwo && id >= p.first_tensor_blocks) {  // the extra work of the two-tensor arrangement
+                map = &kvmap2;
+                id -= (int)p.first_tensor_blocks;
+            }
             const int row_k = (id * 2 * p.num_kv_heads + g) * 16;
             const int row_v = row_k + p.num_kv_heads * 16;
             mbar_expect_tx(bar, STAGE_BYTES);
 #pragma unroll
             for (int x = 0; x < BOXES; ++x) {
-                tma_load_2d_hint(dst + x * kBoxBytes, &kvmap, 64 * x, row_k, bar, policy);
-                tma_load_2d_hint(dst + TILE_BYTES + x * kBoxBytes, &kvmap, 64 * x, row_v, bar, policy);
+                tma_load_2d_hint(dst + x * kBoxBytes, map, 64 * x, row_k, bar, policy);
+                tma_load_2d_hint(dst + TILE_BYTES + x * kBoxBytes, map, 64 * x, row_v, bar, policy);
             }
         }
     };
@@ -129,11 +140,15 @@ decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const DecodeParam
     float m_run = -INFINITY, l_run = 0.f;
     bool failed = false;
 
+    // Phase parity per stage.  A skipped (invalid) block neither issues a copy nor waits, so the parity of a
+    // stage advances only with the copies that really went through it, not with the iteration count.
+    uint32_t stage_parity = 0;
     int i = 0;
     for (; i < nw; ++i) {
         const int stage = i % kDecodeStages;
         if ((valid_mask >> i) & 1u) {
-            const bool got = mbar_wait(my_bars + 8 * stage, (uint32_t)((i / kDecodeStages) & 1));
+            const bool got = mbar_wait(my_bars + 8 * stage, (stage_parity >> stage) & 1u);
+            stage_parity ^= 1u << stage;
             if (__any_sync(FULL, !got)) {
                 failed = true;
                 break;
@@ -209,9 +224,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const DecodeParam
         // A copy barrier never completed.  Latch the error, give copies still in flight a bounded
         // chance to land (their destination must stay allocated), and contribute nothing.
         if (lane == 0) atomicOr(p.status, EKV_DEV_FLAG_TIMEOUT);
+        stage_parity ^= 1u << (i % kDecodeStages);  // the wait that failed belongs to a copy still outstanding
         for (int j = i; j < nw && j < i + kDecodeStages; ++j)
             if ((valid_mask >> j) & 1u)
-                (void)mbar_wait(my_bars + 8 * (j % kDecodeStages), (uint32_t)((j / kDecodeStages) & 1), 200000000ull);
+                (void)mbar_wait(my_bars + 8 * (j % kDecodeStages), (stage_parity >> (j % kDecodeStages)) & 1u, 200000000ull);
         m_run = -INFINITY;
         l_run = 0.f;
 #pragma unroll
@@ -319,25 +335,31 @@ static size_t decode_workspace_need(const ekv_pool *pool, int B, int nsplit) {
     return ml + parts * pool->desc.head_dim * sizeof(float);
 }
 
-template <int D>
-static ekv_status_t launch_decode(ekv_pool *pool, int layer, const DecodeParams &p, int B, cudaStream_t stream) {
+template <int D, bool kTwo>
+static ekv_status_t launch_decode_impl(ekv_pool *pool, const CUtensorMap &map, const CUtensorMap &map2, const DecodeParams &p, int B,
+                                      cudaStream_t stream) {
     constexpr int STAGE_BYTES = 2 * (D / 64) * kBoxBytes;
     const int smem = kDecodeWarps * kDecodeStages * STAGE_BYTES + 1024 + kDecodeWarps * kDecodeStages * 8;
     static bool attr_set[64] = {false};
     const int dev = pool->desc.device;
     if (dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<D, kTwo>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode: shared-memory attribute");
         if (dev < 64) attr_set[dev] = true;
     }
     dim3 grid(p.nsplit, pool->desc.num_kv_heads, B);
-    decode_split_kernel<D><<<grid, kDecodeWarps * 32, smem, stream>>>(pool->kv_map[layer], p);
+    decode_split_kernel<D, kTwo><<<grid, kDecodeWarps * 32, smem, stream>>>(map, map2, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode: split launch");
     decode_combine_kernel<D><<<B * pool->desc.num_q_heads, D, 0, stream>>>(p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode: combine launch");
     return EKV_OK;
+}
+
+template <int D>
+static ekv_status_t launch_decode(ekv_pool *pool, int layer, const DecodeParams &p, int B, cudaStream_t stream) {
+    return launch_decode_impl<D, false>(pool, pool->kv_map[layer], pool->kv_map[layer], p, B, stream);
 }
 
 }  // namespace ekv
@@ -391,6 +413,7 @@ extern "C" ekv_status_t ekv_attn_decode(ekv_pool_t *pool, int32_t layer, const v
     p.chunk_tokens = plan.chunk_tokens;
     p.nsplit = plan.nsplit;
     p.scale_log2 = scale * 1.4426950408889634f;
+    p.first_tensor_blocks = p.total_blocks = 0;
     if (pool->desc.head_dim == 128) return launch_decode<128>(pool, layer, p, B, (cudaStream_t)stream);
     return launch_decode<64>(pool, layer, p, B, (cudaStream_t)stream);
 }
@@ -473,6 +496,67 @@ extern "C" ekv_status_t ekv_attn_decode_static_scratch(ekv_pool_t *pool, int32_t
     p.chunk_tokens = plan.chunk_tokens;
     p.nsplit = plan.nsplit;
     p.scale_log2 = scale * 1.4426950408889634f;
+    p.first_tensor_blocks = p.total_blocks = 0;
     if (pool->desc.head_dim == 128) return launch_decode<128>(pool, layer, p, B, (cudaStream_t)stream);
     return launch_decode<64>(pool, layer, p, B, (cudaStream_t)stream);
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// The two-tensor alternative (paper, "The contiguity constraint": split the KV into two tensors and
+// rewrite the kernel to read both -- prototyped there and rejected).  Built here only to put a number on
+// what the single-range design avoids: the same split kernel with a second tensor map and a per-block
+// choice between the two.
+// ------------------------------------------------------------------------------------------------
+extern "C" ekv_status_t ekv_attn_decode_two_tensor(ekv_pool_t *pool, int32_t layer, const void *second_tensor,
+                                                   int64_t second_blocks, const void *q, void *out, const int32_t *block_tables,
+                                                   int32_t max_blocks_per_seq, const int32_t *seq_lens, int32_t B, float scale,
+                                                   void *workspace, size_t workspace_bytes, void *stream) {
+    ekv_status_t st = check_compute(pool, layer, "ekv_attn_decode_two_tensor");
+    if (st != EKV_OK) return st;
+    if (B < 0 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26) || B > 65535 || second_blocks < 1 || !second_tensor ||
+        ((uintptr_t)second_tensor & 15) || (B > 0 && (!q || !out || !block_tables || !seq_lens)) || ((uintptr_t)q & 15) ||
+        ((uintptr_t)out & 15)) {
+        set_error("ekv_attn_decode_two_tensor: bad argument (B=%d, max_blocks_per_seq=%d, second_blocks=%lld)", B, max_blocks_per_seq,
+                  (long long)second_blocks);
+        return EKV_ERR_INVALID;
+    }
+    if (B == 0) return EKV_OK;
+    const uint64_t rows2 = (uint64_t)second_blocks * 2ull * pool->desc.num_kv_heads * pool->desc.block_size;
+    if (rows2 >= (1ull << 31)) {
+        set_error("ekv_attn_decode_two_tensor: second tensor too large");
+        return EKV_ERR_INVALID;
+    }
+    const DecodePlan plan = plan_decode(pool, B, max_blocks_per_seq);
+    const size_t need = decode_workspace_need(pool, B, plan.nsplit);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) {
+        set_error("ekv_attn_decode_two_tensor: workspace %p of %zu bytes; need %zu bytes, 256-byte aligned", workspace,
+                  workspace_bytes, need);
+        return EKV_ERR_WORKSPACE;
+    }
+    CUtensorMap map2;
+    st = encode_kv_map(const_cast<void *>(second_tensor), rows2, pool->desc.head_dim, pool->desc.block_size, &map2);
+    if (st != EKV_OK) return st;
+    const size_t parts = (size_t)B * pool->desc.num_q_heads * plan.nsplit;
+    DecodeParams p;
+    p.q = (const __nv_bfloat16 *)q;
+    p.block_tables = block_tables;
+    p.seq_lens = seq_lens;
+    p.live = pool->d_live;
+    p.status = pool->d_status;
+    p.part_ml = (float2 *)workspace;
+    p.part_o = (float *)((uint8_t *)workspace + (parts * sizeof(float2) + 255) / 256 * 256);
+    p.out = (__nv_bfloat16 *)out;
+    p.max_blocks = max_blocks_per_seq;
+    p.num_q_heads = pool->desc.num_q_heads;
+    p.num_kv_heads = pool->desc.num_kv_heads;
+    p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
+    p.chunk_tokens = plan.chunk_tokens;
+    p.nsplit = plan.nsplit;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.first_tensor_blocks = pool->base_blocks;  // the first tensor is the pool's base range, whatever the elastic state
+    p.total_blocks = pool->base_blocks + second_blocks;
+    if (pool->desc.head_dim == 128)
+        return launch_decode_impl<128, true>(pool, pool->kv_map[layer], map2, p, B, (cudaStream_t)stream);
+    return launch_decode_impl<64, true>(pool, pool->kv_map[layer], map2, p, B, (cudaStream_t)stream);
 }

@@ -52,4 +52,7 @@ DecodePlan plan_decode(const ekv_pool *pool, int B, int max_blocks_per_seq);
 
 ekv_status_t launch_set_live(ekv_pool *pool, long long value, cudaStream_t stream);
 
+// Tensor map over a KV tensor laid out like a layer range (box 64 channels x block_size tokens, 128-byte swizzle).
+ekv_status_t encode_kv_map(void *base, uint64_t rows, int head_dim, int block_size, CUtensorMap *out);
+
 }  // namespace ekv

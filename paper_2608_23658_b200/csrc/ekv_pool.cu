@@ -172,6 +172,24 @@ ekv_status_t check_compute(ekv_pool *pool, int32_t layer, const char *who) {
     return EKV_OK;
 }
 
+// 2-D view [rows of head_dim bf16] of a KV tensor: box = 64 channels x block_size tokens, 128-byte swizzle.
+ekv_status_t encode_kv_map(void *base, uint64_t rows, int head_dim, int block_size, CUtensorMap *out) {
+    if (!load_driver()) return EKV_ERR_CUDA;
+    cuuint64_t gdim[2] = {(cuuint64_t)head_dim, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)head_dim * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)block_size};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_drv.encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled failed (CUresult %d) for a KV tensor at %p with %llu rows", (int)r, base,
+                  (unsigned long long)rows);
+        return EKV_ERR_CUDA;
+    }
+    return EKV_OK;
+}
+
 static uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
 
 static double now_ms() {
@@ -398,18 +416,8 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
         // and the map never changes when the elastic slice is mapped or unmapped.
         for (int l = 0; l < d.num_layers && st == EKV_OK; ++l) {
             CUtensorMap m;
-            cuuint64_t gdim[2] = {(cuuint64_t)d.head_dim, (cuuint64_t)rows};
-            cuuint64_t gstride[1] = {(cuuint64_t)d.head_dim * 2};
-            cuuint32_t box[2] = {64, (cuuint32_t)d.block_size};
-            cuuint32_t estr[2] = {1, 1};
-            CUresult r = g_drv.encode_tiled(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)p->va[l], gdim, gstride, box,
-                                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            if (r != CUDA_SUCCESS) {
-                set_error("ekv_pool_create: cuTensorMapEncodeTiled failed at layer %d (CUresult %d)", l, (int)r);
-                st = EKV_ERR_CUDA;
-                break;
-            }
+            st = encode_kv_map((void *)p->va[l], rows, d.head_dim, d.block_size, &m);
+            if (st != EKV_OK) break;
             p->kv_map.push_back(m);
         }
     }

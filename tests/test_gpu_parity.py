@@ -253,6 +253,33 @@ def test_decode_out_of_range_block_id_is_skipped_and_latched():
         assert torch.equal(pool.attn_decode(0, q.to(DEV), case.d_tables, case.d_lengths, 0.088), good)
     finally:
         pool.close()
+    # long sequences: every warp walks many blocks, so the stage a skipped block would have used is reused
+    pool = make_pool(shape, 512, 32, grown=False)
+    try:
+        lengths = [3000, 2500]
+        case = Case(shape, lengths, 512, 53, pool=pool)
+        q = rand_q(54, 2, shape)
+        bad = case.tables.clone()
+        skip = [0, 5, 6, 40, 187]                               # first block, neighbours, middle, the last one
+        for j in skip:
+            bad[0, j] = 530
+        out = pool.attn_decode(0, q.to(DEV), bad.to(DEV), case.d_lengths, 0.088)
+        torch.cuda.synchronize()
+        assert pool.poll_status() == ekv.Status.ERR_BLOCK_OOB   # and not a timeout
+        K, V = case.seqs[0]
+        keep = torch.tensor([t for t in range(3000) if t // 16 not in skip])
+        nb = (len(keep) + 15) // 16
+        host = empty_cache(nb, shape)
+        tbl = torch.arange(nb, dtype=torch.int32)[None]
+        place_sequence(host, shape, tbl[0], K[keep], V[keep])
+        want = oracle.attn_decode(host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q[:1], tbl,
+                                  torch.tensor([len(keep)]), 0.088)
+        check_close(out[:1], want, "long decode with skipped blocks")
+        good = pool.attn_decode(0, q.to(DEV), case.d_tables, case.d_lengths, 0.088)
+        check_close(good, case.oracle_decode(q, 0.088), "long decode")
+        assert torch.equal(out[1], good[1])
+    finally:
+        pool.close()
 
 
 def test_decode_argument_errors():
