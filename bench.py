@@ -365,6 +365,45 @@ def measure_toggle(device, cycles=5):
     return out
 
 
+def measure_decode_long_context(device, peaks, reps=5):
+    """Decode attention on the configs[3] batch (64 sequences, 64q/8kv heads, contexts U[32768,131072], 21.3 GB of KV
+    per launch) in a pool just large enough for it."""
+    import paper_2608_23658_b200 as ekv
+    cfg, s = I.C4, I.C4.shape
+    lengths = I.decode_lengths(cfg)
+    need = int(I.blocks_for(lengths, s.block_size).sum())
+    elastic = int(need * 1.02 * cfg.elastic_fraction)
+    pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim,
+                    base_blocks=int(need * 1.02) - elastic, elastic_blocks=elastic, start_grown=True, device=device.index or 0)
+    try:
+        live = pool.info.live_blocks
+        tables, _ = I.assign_blocks(cfg.seed, 12, lengths, s.block_size, live)
+        I.fill_pool_layer_(pool.layer_tensor(0), cfg.seed, chunk=1 << 26)
+        B = len(lengths)
+        q = I.normal_bf16(cfg.seed, 3, 0, B * s.num_q_heads * s.head_dim, device=device).view(B, s.num_q_heads, s.head_dim)
+        d_tables, d_lens = tables.to(device), lengths.to(torch.int32).to(device)
+        ws = pool.workspace(B, int(tables.shape[1]) * s.block_size)
+        out = torch.empty_like(q)
+        scale = 1.0 / math.sqrt(s.head_dim)
+        for _ in range(3):
+            pool.attn_decode(0, q, d_tables, d_lens, scale, out=out, workspace=ws)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            pool.attn_decode(0, q, d_tables, d_lens, scale, out=out, workspace=ws)
+        e1.record()
+        torch.cuda.synchronize(device)
+        ms = e0.elapsed_time(e1) / reps
+        nbytes = I.decode_algorithmic_bytes(lengths, s)
+        gbs = nbytes / ms / 1e6
+        return {"ms": round(ms, 3), "gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
+                "frac_of_nominal_8000": round(gbs / 8000.0, 4), "algorithmic_bytes": nbytes,
+                "elastic_fraction_of_blocks": round(elastic / live, 3),
+                "workload": "c4 decode: 64 seqs, 64q/8kv heads d128, contexts U[32768,131072]"}
+    finally:
+        pool.close()
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 
 
@@ -406,7 +445,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(1e3 * total / args.steps, 3),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "sample": sample},
+            "config": {"workload": cfg.name, "batch": cfg.decode.batch, "heads": "32q/8kv", "head_dim": 128, "block_size": 16,
+                       "step": "oracle attn_decode on a sample of the workload's sequences", "sample": sample},
             "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -528,6 +568,8 @@ def main():
         line["prefill"] = measure_prefill(device, peaks)
         torch.cuda.empty_cache()
         line["toggle"] = measure_toggle(device)
+        torch.cuda.empty_cache()
+        line["decode_long_context"] = measure_decode_long_context(device, peaks)
         one, nbytes, sample, cores = oracle_decode_sample(cfg)
         one()
         reps, t = 0, 0.0

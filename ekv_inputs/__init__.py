@@ -220,11 +220,11 @@ def decode_lengths(cfg: Config, batch: int | None = None) -> torch.Tensor:
 KV_STREAM = 21  # stream id of "pool content as a function of the physical element index"
 
 
-def fill_pool_layer_(layer_view: torch.Tensor, seed: int, layer: int = 0, first_block: int = 0) -> None:
+def fill_pool_layer_(layer_view: torch.Tensor, seed: int, layer: int = 0, first_block: int = 0, chunk: int = 1 << 24) -> None:
     """Fill a [blocks, 2, Hkv, bs, d] bf16 view of a layer (starting at physical block first_block)
     so that element e of the layer holds normal_bf16(seed, KV_STREAM + layer, e)."""
     block_elems = layer_view[0].numel()
-    fill_normal_bf16_(layer_view, seed, KV_STREAM + layer, start=first_block * block_elems)
+    fill_normal_bf16_(layer_view, seed, KV_STREAM + layer, start=first_block * block_elems, chunk=chunk)
 
 
 def host_blocks(seed: int, layer: int, block_ids, block_elems: int) -> torch.Tensor:

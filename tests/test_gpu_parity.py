@@ -494,3 +494,60 @@ def test_prefill_edge_cases_bad_ids_empty_requests_and_both_kernels_agree():
             outs[impl] = torch.load(path)
         diff = (outs["mma"].float() - outs["tc"].float()).abs()
         assert diff.max().item() <= MAX_ABS and diff.mean().item() <= MEAN_ABS
+
+
+def test_recommit_out_of_memory_leaves_the_pool_shrunk_and_usable():
+    """The paper's recommit OOM (the memory lent back may be gone when the controller wants it again): a grow
+    whose physical allocation cannot be satisfied returns EKV_ERR_OOM, the pool stays shrunk, and attention over
+    base blocks is unaffected.  The elastic range asked for is larger than the whole device, so creation fails at
+    once without filling the memory."""
+    shape = I.LLAMA8B
+    total = torch.cuda.mem_get_info()[1]
+    huge_blocks = int(2 * total // shape.block_bytes)
+    pool = make_pool(shape, 128, huge_blocks, grown=False)        # reserving address space costs no memory
+    try:
+        case = Case(shape, [500, 70], 128, 95, pool=pool)
+        q = rand_q(96, 2, shape)
+        ref = case.decode(q, 0.088)
+        free0 = torch.cuda.mem_get_info()[0]
+        with pytest.raises(ekv.EkvError) as e:
+            pool.grow()
+        assert e.value.status == ekv.Status.ERR_OOM
+        info = pool.info
+        assert not info.grown and not info.physical_held and info.live_blocks == info.base_blocks
+        assert abs(torch.cuda.mem_get_info()[0] - free0) < (64 << 20)   # nothing left allocated
+        assert torch.equal(case.decode(q, 0.088), ref)
+        assert pool.poll_status() == ekv.Status.OK
+    finally:
+        pool.close()
+    with pytest.raises(ekv.EkvError) as e:                       # a base range that cannot be backed: nothing is left behind
+        make_pool(shape, huge_blocks, 0)
+    assert e.value.status == ekv.Status.ERR_OOM
+
+
+def test_empty_calls_are_no_ops():
+    """T = 0, B = 0 and R = 0 are legal and launch nothing."""
+    shape = I.LLAMA8B
+    pool = make_pool(shape, 64)
+    try:
+        view = pool.layer_tensor(0)
+        view.view(torch.int16).fill_(0x3C00)
+        before = view.cpu()
+        z_kv = torch.empty(0, shape.num_kv_heads, shape.head_dim, dtype=torch.bfloat16, device=DEV)
+        pool.write_kv(0, z_kv, z_kv, torch.empty(0, dtype=torch.int64, device=DEV))
+        z_q = torch.empty(0, shape.num_q_heads, shape.head_dim, dtype=torch.bfloat16, device=DEV)
+        out = pool.attn_decode(0, z_q, torch.empty(0, 4, dtype=torch.int32, device=DEV),
+                               torch.empty(0, dtype=torch.int32, device=DEV), 0.1,
+                               workspace=torch.empty(256, dtype=torch.uint8, device=DEV))
+        assert out.shape == z_q.shape
+        cu = torch.zeros(1, dtype=torch.int32)
+        outp = pool.attn_prefill_chunk(0, z_q, torch.empty(0, 4, dtype=torch.int32, device=DEV), cu.to(DEV), cu,
+                                       torch.empty(0, dtype=torch.int32, device=DEV), 0.1)
+        assert outp.shape == z_q.shape
+        ekv.ekv_move_blocks(pool.handle, torch.empty(0, dtype=torch.int32, device=DEV),
+                            torch.empty(0, dtype=torch.int32, device=DEV))
+        torch.cuda.synchronize()
+        assert pool.poll_status() == ekv.Status.OK
+        assert torch.equal(view.cpu(), before)
+    finally:
+        pool.close()
