@@ -39,7 +39,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) per algorithmic byte of the decode split kernel, from the ncu capture
 # summarised in profiles/decode_split_c2_batch32.md (a 32-sequence slice of the same workload; the
 # traffic is proportional to the KV bytes read, so it is scaled to the full launch by that ratio).
-DECODE_SPLIT_DRAM_TRAFFIC_RATIO = (623.645952 + 5.713408) / 622.920860
+DECODE_SPLIT_DRAM_TRAFFIC_RATIO = (623.649792 + 4.772352) / 622.920860
 
 
 def measured_peaks():
@@ -551,7 +551,7 @@ def main():
                    "context_tokens": int(wl.lengths.sum()), "step": "ekv_write_kv + ekv_attn_decode (split + combine)",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2 (%.2f GB of KV per step)" % (wl.decode_bytes / 1e9)},
-        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel<128> + decode_combine_kernel<128>",
+        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel<128, false> + decode_combine_kernel<128>",
                      "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": round(achieved / peaks["hbm_gbs"], 4), "peak_kind": f"{peaks_kind} copy bandwidth",
                      "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": int(DECODE_SPLIT_DRAM_TRAFFIC_RATIO * wl.decode_bytes),
