@@ -159,33 +159,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
 #define EKV_TRACE_FLUSH do { } while (0)
 #endif
 
-#ifndef EKV_TC_PART
-#define EKV_TC_PART 6
-#endif
-#ifndef EKV_TC_EMU
-#define EKV_TC_EMU 0
-#endif
-static constexpr int kPartSteps = EKV_TC_PART;  // PV k-steps (16 keys each) covered by the early P_PART arrival (even, 2..6)
-static constexpr int kEmulatePairsOf8 = EKV_TC_EMU;  // of every 8 pairs of exponentials, how many go to the FMA pipe instead of the MUFU pipe
-
-// 2^x for a pair on the FMA pipe: x = n + f with n = round(x), f in [-0.5, 0.5]; cubic minimax of 2^f
-// (max relative error 7.5e-5, far below the bf16 rounding P gets anyway); 2^n goes into the exponent
-// field by an integer add.  Inputs at or below -126 (masked scores arrive as -inf) return ~1e-38.
-__device__ __forceinline__ float2 exp2_fma_pair(float2 x) {
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 magic = make_float2(12582912.f, 12582912.f);  // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
-    const float2 t = __fadd2_rn(x, magic);
-    const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
-    float2 q = __ffma2_rn(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.2426111251f, 0.2426111251f));
-    q = __ffma2_rn(q, f, make_float2(0.6932609677f, 0.6932609677f));
-    q = __ffma2_rn(q, f, make_float2(0.9999280572f, 0.9999280572f));
-    float2 r;
-    r.x = __uint_as_float(__float_as_uint(q.x) + (__float_as_uint(t.x) << 23));
-    r.y = __uint_as_float(__float_as_uint(q.y) + (__float_as_uint(t.y) << 23));
-    return r;
-}
+static constexpr int kPartSteps = 6;  // PV k-steps (16 keys each) covered by the early P_PART arrival (even, 2..6)
 
 struct Shared {
     uint32_t base;      // shared-window address of the aligned base
@@ -527,8 +501,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             const float m_use = m_run > -INFINITY ? m_run : 0.f;
             // ---- P = exp2(S*scale - m) (a masked -inf gives 0), row sum, bf16 pairs into the S columns
             // P of the first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
-            // (EKV_TC_EMU=1 evaluates every second pair of exponentials on the FMA pipe instead of the MUFU
-            // pipe; measured slower on B200 under the 1 kW power cap -- 1.10 vs 1.20-1.25 PFLOP/s -- so off.)
             float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
             const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
 #pragma unroll
@@ -539,9 +511,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                     const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
                     const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
                     const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
-                    // pairs are numbered i/2 (MUFU first) and i/2+1; the second one of a group is emulated while the
-                    // group index (i/4 of 8) is below the configured count
-                    const float2 pb = ((i >> 2) < kEmulatePairsOf8) ? exp2_fma_pair(xb) : make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+                    const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
                     acc_a = __fadd2_rn(acc_a, pa);
                     acc_b = __fadd2_rn(acc_b, pb);
                     pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
