@@ -20,3 +20,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """Build (or refresh) libekv.so and the oracle once per session; both builds are no-ops when up to date.
+    The library itself never builds or falls back on its own: a missing libekv.so is a loud ImportError."""
+    from paper_2608_23658_b200 import build as ekv_build
+    ekv_build.build()
+    import oracle
+    oracle.build()
