@@ -277,8 +277,31 @@ decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const __grid_cons
     }
 }
 
+// Block-wide max / sum over D threads (D = 64 or 128), fixed order: bitwise reproducible.
+template <int D, bool kMax>
+__device__ __forceinline__ float block_reduce(float v, float *scratch) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float u = __shfl_xor_sync(0xffffffffu, v, o);
+        v = kMax ? fmaxf(v, u) : v + u;
+    }
+    __syncthreads();  // scratch may still be read from an earlier reduction
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = scratch[0];
+#pragma unroll
+    for (int w = 1; w < D / 32; ++w) r = kMax ? fmaxf(r, scratch[w]) : r + scratch[w];
+    return r;
+}
+
+// One CTA per (sequence, q-head), one thread per output channel.  The splits are walked in parallel: the
+// statistics (m, l) are reduced across the block, and the weighted sum of partial rows is taken in tiles of D
+// splits whose weights sit in shared memory, so that a long sequence with hundreds of splits costs a few
+// rounds of independent loads instead of hundreds of dependent ones.
 template <int D>
 __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeParams p) {
+    __shared__ float scratch[D / 32];
+    __shared__ float w_tile[D];
     const int bh = blockIdx.x;
     const int b = bh / p.num_q_heads;
     const int x = threadIdx.x;
@@ -287,17 +310,37 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeParams p)
     const int ns = (L + p.chunk_tokens - 1) / p.chunk_tokens;
     const float2 *ml = p.part_ml + (size_t)bh * p.nsplit;
     const float *po = p.part_o + (size_t)bh * p.nsplit * D;
-    float mstar = -INFINITY;
-    for (int s = 0; s < ns; ++s) mstar = fmaxf(mstar, ml[s].x);
-    float acc = 0.f, lsum = 0.f;
-    if (mstar > -INFINITY) {
-        for (int s = 0; s < ns; ++s) {
-            const float2 v = ml[s];
-            const float w = (v.x > -INFINITY) ? fast_exp2(v.x - mstar) : 0.f;
-            lsum += w * v.y;
-            acc += w * po[(size_t)s * D + x];
+    float mloc = -INFINITY;
+    for (int s = x; s < ns; s += D) mloc = fmaxf(mloc, ml[s].x);
+    const float mstar = block_reduce<D, true>(mloc, scratch);
+    float acc = 0.f, lloc = 0.f;
+    if (mstar > -INFINITY) {  // block-uniform
+        for (int s0 = 0; s0 < ns; s0 += D) {
+            const int s = s0 + x;
+            float w = 0.f;
+            if (s < ns) {
+                const float2 v = ml[s];
+                w = (v.x > -INFINITY) ? fast_exp2(v.x - mstar) : 0.f;
+                lloc += w * v.y;
+            }
+            __syncthreads();  // the previous tile's weights are no longer needed
+            w_tile[x] = w;
+            __syncthreads();
+            const int n = min(D, ns - s0);
+            const float *src = po + (size_t)s0 * D + x;
+            int i = 0;
+            for (; i + 4 <= n; i += 4) {
+                const float o0 = src[(size_t)i * D], o1 = src[(size_t)(i + 1) * D];
+                const float o2 = src[(size_t)(i + 2) * D], o3 = src[(size_t)(i + 3) * D];
+                acc += w_tile[i] * o0;
+                acc += w_tile[i + 1] * o1;
+                acc += w_tile[i + 2] * o2;
+                acc += w_tile[i + 3] * o3;
+            }
+            for (; i < n; ++i) acc += w_tile[i] * src[(size_t)i * D];
         }
     }
+    const float lsum = block_reduce<D, false>(lloc, scratch);
     p.out[(size_t)bh * D + x] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
 }
 
@@ -321,7 +364,9 @@ DecodePlan plan_decode(const ekv_pool *pool, int B, int max_blocks_per_seq) {
     chunk = (chunk + 63) / 64 * 64;
     const int cmax = chunk_max_tokens();
     if (chunk > cmax) chunk = cmax;
-    if (chunk < 64) chunk = 64;
+    // at least 4 blocks per warp (256 keys) when the length allows: below that the fixed cost of a CTA dominates
+    const long long cmin = max_len >= 256 ? 256 : (max_len + 63) / 64 * 64;
+    if (chunk < cmin) chunk = cmin;
     DecodePlan plan;
     plan.chunk_tokens = (int)chunk;
     plan.nsplit = (int)((max_len + chunk - 1) / chunk);
