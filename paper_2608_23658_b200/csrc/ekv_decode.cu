@@ -66,7 +66,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const __grid_cons
     int L = p.seq_lens[b];
     L = max(0, min(L, p.max_blocks * 16));
     const int t_begin = split * p.chunk_tokens;
-    if (t_begin >= L) return;  // whole CTA leaves before any barrier exists
+    if (t_begin >= L) {  // whole CTA leaves before any barrier exists
+        if (p.nsplit == 1)  // no combine pass will run: an empty sequence gets its zero rows here
+            for (int e = threadIdx.x; e < p.group * D; e += kDecodeWarps * 32)
+                p.out[((size_t)b * p.num_q_heads + (size_t)g * p.group) * D + e] = __float2bfloat16_rn(0.f);
+        return;
+    }
     const int t_end = min(L, t_begin + p.chunk_tokens);
     const int nblk = (t_end - t_begin + 15) >> 4;
     const int nw = max(0, (nblk - warp + kDecodeWarps - 1) / kDecodeWarps);  // blocks this warp owns (<= 32)
@@ -272,8 +277,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const __grid_cons
             }
         }
         const size_t slot = ((size_t)b * p.num_q_heads + (size_t)g * p.group + h) * p.nsplit + split;
-        p.part_o[slot * D + x] = acc;
-        if (x == 0) p.part_ml[slot] = make_float2(mstar, lsum);
+        if (p.nsplit == 1) {  // the only split of every sequence: finish here, no partials, no combine pass
+            p.out[slot * D + x] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
+        } else {
+            p.part_o[slot * D + x] = acc;
+            if (x == 0) p.part_ml[slot] = make_float2(mstar, lsum);
+        }
     }
 }
 
@@ -396,6 +405,7 @@ static ekv_status_t launch_decode_impl(ekv_pool *pool, const CUtensorMap &map, c
     decode_split_kernel<D, kTwo><<<grid, kDecodeWarps * 32, smem, stream>>>(map, map2, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode: split launch");
+    if (p.nsplit == 1) return EKV_OK;  // the split kernel wrote the final rows itself
     decode_combine_kernel<D><<<B * pool->desc.num_q_heads, D, 0, stream>>>(p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_decode: combine launch");

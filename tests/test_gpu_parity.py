@@ -551,3 +551,23 @@ def test_empty_calls_are_no_ops():
         assert torch.equal(view.cpu(), before)
     finally:
         pool.close()
+
+
+def test_decode_single_split_path_writes_final_rows_directly():
+    """Many short sequences: one key range per sequence, so the split kernel finishes the rows itself (no combine
+    pass).  Includes empty sequences, which must still come out as zero rows."""
+    shape = I.LLAMA8B
+    lengths = [int(x) for x in I.uniform_ints(97, 11, 200, 0, 500)]
+    lengths[3] = 0
+    lengths[77] = 0
+    need = int(I.blocks_for(torch.tensor(lengths), 16).sum())
+    case = Case(shape, lengths, need + 8, 97, max_blocks_per_seq=32)   # 32 blocks = 512 keys = one range
+    try:
+        q = rand_q(98, len(lengths), shape)
+        out = torch.full((len(lengths), shape.num_q_heads, shape.head_dim), float("nan"), dtype=torch.bfloat16, device=DEV)
+        case.pool.attn_decode(0, q.to(DEV), case.d_tables, case.d_lengths, 0.088, out=out)
+        check_close(out, case.oracle_decode(q, 0.088), "single-split decode")
+        assert (out[3] == 0).all() and (out[77] == 0).all()
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
