@@ -365,6 +365,42 @@ def measure_toggle(device, cycles=5):
     return out
 
 
+def measure_write_kv(device, peaks):
+    """ekv_write_kv bandwidth at the chunk sizes of configs[2] (8192 and 32768 tokens), L2 flushed between reps."""
+    import paper_2608_23658_b200 as ekv
+    s = I.C3.shape
+    res = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    for T in (8192, 32768):
+        pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=T // 16 + 64,
+                        device=device.index or 0)
+        try:
+            live = pool.info.live_blocks
+            slots = (I.permutation(I.C3.seed, 14, live)[:T // 16].repeat_interleave(16) * 16 + torch.arange(T) % 16).to(device)
+            n = T * s.num_kv_heads * s.head_dim
+            k = I.normal_bf16(I.C3.seed, 7, 0, n, device=device).view(T, s.num_kv_heads, s.head_dim)
+            v = I.normal_bf16(I.C3.seed, 8, 0, n, device=device).view(T, s.num_kv_heads, s.head_dim)
+            for _ in range(3):
+                pool.write_kv(0, k, v, slots)
+            ts = []
+            for _ in range(7):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                pool.write_kv(0, k, v, slots)
+                e1.record()
+                torch.cuda.synchronize(device)
+                ts.append(e0.elapsed_time(e1))
+            ms = statistics.median(ts)
+            gbs = I.write_algorithmic_bytes(T, s) / ms / 1e6
+            res[f"tokens_{T}"] = {"ms": round(ms, 4), "gbs_read_plus_write": round(gbs, 1),
+                                  "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}
+        finally:
+            pool.close()
+    res["workload"] = "slot-mapped write of K and V rows, 8 kv heads x 128 channels, blocks scattered over the pool"
+    return res
+
+
 def measure_decode_long_context(device, peaks, reps=5):
     """Decode attention on the configs[3] batch (64 sequences, 64q/8kv heads, contexts U[32768,131072], 21.3 GB of KV
     per launch) in a pool just large enough for it."""
@@ -570,6 +606,7 @@ def main():
         line["toggle"] = measure_toggle(device)
         torch.cuda.empty_cache()
         line["decode_long_context"] = measure_decode_long_context(device, peaks)
+        line["write_kv"] = measure_write_kv(device, peaks)
         one, nbytes, sample, cores = oracle_decode_sample(cfg)
         one()
         reps, t = 0, 0.0
