@@ -29,10 +29,20 @@
  * KV layout (part of the boundary).  All layers share one geometry.  From ekv_layer_ptr(layer),
  * channel x of token-in-block t of kv-head h of the K (kv=0) or V (kv=1) half of physical block n
  * is the bf16 at byte offset
- *       ((((n*2 + kv)*num_kv_heads + h)*block_size + t)*head_dim + x) * 2 .
- * Block n therefore occupies bytes [n*block_bytes, (n+1)*block_bytes); blocks 0..base_blocks-1
- * are backed by the base handle, blocks base_blocks..base_blocks+elastic_blocks-1 by the elastic
- * handle.  A slot is block*block_size + t.
+ *       n*block_stride_bytes + ((((kv*num_kv_heads + h)*block_size + t)*head_dim + x) * 2 ,
+ * with block_stride_bytes = block_bytes = 2*num_kv_heads*block_size*head_dim*2 by default: block n of
+ * a layer occupies bytes [n*block_bytes, (n+1)*block_bytes) of that layer's own range.  Blocks
+ * 0..base_blocks-1 are backed by the base handle, blocks base_blocks..base_blocks+elastic_blocks-1
+ * by the elastic handle.  A slot is block*block_size + t.
+ *
+ * EKV_FUSED_RANGE (this build's variation on the paper's arrangement, for a cheaper toggle): the
+ * driver's map / unmap / set-access cost is per call, not per byte, and one call per layer is what
+ * makes a toggle take milliseconds.  With this flag the pool reserves ONE range for the whole model
+ * and interleaves the layers inside every block id: block n of layer l lives at
+ * (n*num_layers + l)*block_bytes, i.e. ekv_layer_ptr(l) = range + l*block_bytes and
+ * block_stride_bytes = num_layers*block_bytes.  Every layer is still ONE pointer indexed by block
+ * id (a strided tensor instead of a dense one), the elastic block ids are still the top of the
+ * range, and grow / shrink are one map / unmap for all layers.  The kernels are the same code.
  */
 #ifndef EKV_H_
 #define EKV_H_
@@ -68,8 +78,10 @@ enum { EKV_BF16 = 0 };
 /* flag bits */
 enum {
     EKV_START_GROWN = 1u << 0,   /* ekv_pool_create: map the elastic slice right away */
-    EKV_KEEP_PHYSICAL = 1u << 1  /* ekv_shrink: unmap only, keep the elastic handle (bytes survive
+    EKV_KEEP_PHYSICAL = 1u << 1, /* ekv_shrink: unmap only, keep the elastic handle (bytes survive
                                     until the next ekv_grow maps it again) */
+    EKV_FUSED_RANGE = 1u << 2    /* ekv_pool_create: ONE virtual range and two handles for all layers
+                                    instead of one range and two handles per layer (see below) */
 };
 
 typedef struct ekv_pool_desc {
@@ -96,7 +108,9 @@ typedef struct ekv_pool_info {
     int32_t grown;           /* elastic slice mapped */
     int32_t physical_held;   /* elastic handles exist (mapped, or kept by EKV_KEEP_PHYSICAL) */
     int32_t num_layers;
-    int32_t reserved;
+    int32_t num_ranges;          /* virtual ranges the pool holds: num_layers, or 1 with EKV_FUSED_RANGE */
+    uint64_t block_stride_bytes; /* distance between consecutive block ids of one layer: block_bytes, or
+                                    num_layers*block_bytes with EKV_FUSED_RANGE */
 } ekv_pool_info_t;
 
 /*

@@ -12,6 +12,7 @@ _lib = None
 EKV_BF16 = 0
 EKV_START_GROWN = 1
 EKV_KEEP_PHYSICAL = 2
+EKV_FUSED_RANGE = 4
 
 
 class Status(enum.IntEnum):
@@ -60,7 +61,7 @@ class PoolInfo(ctypes.Structure):
     _fields_ = [("granularity", ctypes.c_uint64), ("block_bytes", ctypes.c_uint64), ("base_bytes", ctypes.c_uint64),
                 ("elastic_bytes", ctypes.c_uint64), ("base_blocks", ctypes.c_int64), ("elastic_blocks", ctypes.c_int64),
                 ("live_blocks", ctypes.c_int64), ("grown", ctypes.c_int32), ("physical_held", ctypes.c_int32),
-                ("num_layers", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("num_layers", ctypes.c_int32), ("num_ranges", ctypes.c_int32), ("block_stride_bytes", ctypes.c_uint64)]
 
 
 _u64p = ctypes.POINTER(ctypes.c_uint64)

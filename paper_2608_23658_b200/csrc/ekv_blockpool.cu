@@ -275,8 +275,8 @@ namespace ekv {
 // One CTA per (pair, layer): copies block src -> dst (block_bytes, 16-byte pieces).  HBM-bound copy.
 __global__ void __launch_bounds__(256) move_blocks_kernel(const unsigned long long *__restrict__ layer_base, int num_layers,
                                                           const int *__restrict__ src_ids, const int *__restrict__ dst_ids,
-                                                          int pieces_per_block, const long long *__restrict__ live_ptr,
-                                                          unsigned *status) {
+                                                          int pieces_per_block, long long block_stride_pieces,
+                                                          const long long *__restrict__ live_ptr, unsigned *status) {
     const int pair = blockIdx.x, layer = blockIdx.y;
     const long long live = *live_ptr;
     const long long s = src_ids[pair], d = dst_ids[pair];
@@ -284,8 +284,8 @@ __global__ void __launch_bounds__(256) move_blocks_kernel(const unsigned long lo
         if (threadIdx.x == 0) atomicOr(status, EKV_DEV_FLAG_OOB);
         return;
     }
-    const uint4 *src = reinterpret_cast<const uint4 *>(layer_base[layer]) + s * pieces_per_block;
-    uint4 *dst = reinterpret_cast<uint4 *>(layer_base[layer]) + d * pieces_per_block;
+    const uint4 *src = reinterpret_cast<const uint4 *>(layer_base[layer]) + s * block_stride_pieces;
+    uint4 *dst = reinterpret_cast<uint4 *>(layer_base[layer]) + d * block_stride_pieces;
     for (int i = threadIdx.x; i < pieces_per_block; i += blockDim.x) dst[i] = src[i];
 }
 
@@ -301,7 +301,8 @@ extern "C" ekv_status_t ekv_move_blocks(ekv_pool_t *pool, const int32_t *src_ids
     if (n == 0) return EKV_OK;
     dim3 grid((unsigned)n, (unsigned)pool->desc.num_layers);
     move_blocks_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(pool->d_layer_base, pool->desc.num_layers, src_ids, dst_ids,
-                                                               (int)(pool->block_bytes / 16), pool->d_live, pool->d_status);
+                                                               (int)(pool->block_bytes / 16), (long long)(pool->block_stride / 16),
+                                                               pool->d_live, pool->d_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_move_blocks launch");
     return EKV_OK;

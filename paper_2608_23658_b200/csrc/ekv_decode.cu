@@ -111,13 +111,13 @@ decode_split_kernel(const __grid_constant__ CUtensorMap kvmap, const __grid_cons
                 map = &kvmap2;
                 id -= (int)p.first_tensor_blocks;
             }
-            const int row_k = (id * 2 * p.num_kv_heads + g) * 16;
+            const int row_k = g * 16;  // row inside the block: (K|V, kv-head, token)
             const int row_v = row_k + p.num_kv_heads * 16;
             mbar_expect_tx(bar, STAGE_BYTES);
 #pragma unroll
             for (int x = 0; x < BOXES; ++x) {
-                tma_load_2d_hint(dst + x * kBoxBytes, map, 64 * x, row_k, bar, policy);
-                tma_load_2d_hint(dst + TILE_BYTES + x * kBoxBytes, map, 64 * x, row_v, bar, policy);
+                tma_load_3d_hint(dst + x * kBoxBytes, map, 64 * x, row_k, id, bar, policy);
+                tma_load_3d_hint(dst + TILE_BYTES + x * kBoxBytes, map, 64 * x, row_v, id, bar, policy);
             }
         }
     };
@@ -577,8 +577,7 @@ extern "C" ekv_status_t ekv_attn_decode_two_tensor(ekv_pool_t *pool, int32_t lay
         return EKV_ERR_INVALID;
     }
     if (B == 0) return EKV_OK;
-    const uint64_t rows2 = (uint64_t)second_blocks * 2ull * pool->desc.num_kv_heads * pool->desc.block_size;
-    if (rows2 >= (1ull << 31)) {
+    if (second_blocks >= (1ll << 31)) {
         set_error("ekv_attn_decode_two_tensor: second tensor too large");
         return EKV_ERR_INVALID;
     }
@@ -590,7 +589,8 @@ extern "C" ekv_status_t ekv_attn_decode_two_tensor(ekv_pool_t *pool, int32_t lay
         return EKV_ERR_WORKSPACE;
     }
     CUtensorMap map2;
-    st = encode_kv_map(const_cast<void *>(second_tensor), rows2, pool->desc.head_dim, pool->desc.block_size, &map2);
+    st = encode_kv_map(const_cast<void *>(second_tensor), (uint64_t)second_blocks, pool->block_bytes, pool->desc.num_kv_heads,
+                       pool->desc.head_dim, pool->desc.block_size, &map2);
     if (st != EKV_OK) return st;
     const size_t parts = (size_t)B * pool->desc.num_q_heads * plan.nsplit;
     DecodeParams p;

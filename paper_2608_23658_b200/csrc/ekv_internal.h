@@ -17,21 +17,29 @@ struct ekv_pool {
     ekv_vmm_backend_t be;
     bool host_only;  // created through a replacement VMM backend: no device state, no compute
 
-    uint64_t granularity, block_bytes, base_bytes, elastic_bytes;
-    int64_t base_blocks, elastic_blocks;
+    // A "range" is one virtual address reservation with one base mapping and one elastic mapping.  Default: one
+    // range per layer (the paper's arrangement).  EKV_FUSED_RANGE: a single range for all layers, block n of
+    // layer l at (n*num_layers + l)*block_bytes, so a toggle is one map / unmap instead of one per layer.
+    int num_ranges;
+    bool fused;
+    uint64_t granularity, block_bytes, block_stride;  // block_stride: bytes between consecutive block ids of one layer
+    uint64_t base_bytes, elastic_bytes;               // per RANGE
+    int64_t base_blocks, elastic_blocks;              // per layer
     bool grown;
 
-    std::vector<uint64_t> va;              // per layer: start of the reserved range
-    std::vector<uint64_t> base_handle;     // per layer
-    std::vector<uint64_t> elastic_handle;  // per layer, valid while elastic_held
-    std::vector<char> elastic_held;        // per layer: the elastic handle exists
+    std::vector<uint64_t> va;              // per range: start of the reserved range
+    std::vector<uint64_t> base_handle;     // per range
+    std::vector<uint64_t> elastic_handle;  // per range, valid while elastic_held
+    std::vector<char> elastic_held;        // per range: the elastic handle exists
+
+    uint64_t layer_base(int layer) const { return fused ? va[0] + (uint64_t)layer * block_bytes : va[layer]; }
 
     // device state (absent when host_only)
     long long *d_live;      // device words: [0] number of block ids kernels may dereference, [1] abort word
     unsigned *h_status;     // pinned, host-mapped status word
     unsigned *d_status;     // its device alias
     unsigned long long *d_layer_base;  // device array: start address of every layer's range
-    std::vector<CUtensorMap> kv_map;  // per layer: 2-D view [rows of head_dim bf16], box 64 x block_size, 128B swizzle
+    std::vector<CUtensorMap> kv_map;  // per layer: 3-D view (channel, row in block, block id), box 64 x block_size x 1, 128B swizzle
     int sm_count;
 };
 
@@ -52,7 +60,9 @@ DecodePlan plan_decode(const ekv_pool *pool, int B, int max_blocks_per_seq);
 
 ekv_status_t launch_set_live(ekv_pool *pool, long long value, cudaStream_t stream);
 
-// Tensor map over a KV tensor laid out like a layer range (box 64 channels x block_size tokens, 128-byte swizzle).
-ekv_status_t encode_kv_map(void *base, uint64_t rows, int head_dim, int block_size, CUtensorMap *out);
+// Tensor map over a KV tensor of `blocks` blocks that are `block_stride` bytes apart, each laid out
+// (K|V, kv-head, token, channel): dims (channel, row in block, block), box 64 x block_size x 1, 128-byte swizzle.
+ekv_status_t encode_kv_map(void *base, uint64_t blocks, uint64_t block_stride, int num_kv_heads, int head_dim, int block_size,
+                           CUtensorMap *out);
 
 }  // namespace ekv

@@ -5,6 +5,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <chrono>
 #include <mutex>
 #include <new>
@@ -172,19 +173,19 @@ ekv_status_t check_compute(ekv_pool *pool, int32_t layer, const char *who) {
     return EKV_OK;
 }
 
-// 2-D view [rows of head_dim bf16] of a KV tensor: box = 64 channels x block_size tokens, 128-byte swizzle.
-ekv_status_t encode_kv_map(void *base, uint64_t rows, int head_dim, int block_size, CUtensorMap *out) {
+ekv_status_t encode_kv_map(void *base, uint64_t blocks, uint64_t block_stride, int num_kv_heads, int head_dim, int block_size,
+                           CUtensorMap *out) {
     if (!load_driver()) return EKV_ERR_CUDA;
-    cuuint64_t gdim[2] = {(cuuint64_t)head_dim, (cuuint64_t)rows};
-    cuuint64_t gstride[1] = {(cuuint64_t)head_dim * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)block_size};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_drv.encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
+    cuuint64_t gdim[3] = {(cuuint64_t)head_dim, (cuuint64_t)2 * num_kv_heads * block_size, (cuuint64_t)blocks};
+    cuuint64_t gstride[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)block_stride};
+    cuuint32_t box[3] = {64, (cuuint32_t)block_size, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_drv.encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, gdim, gstride, box, estr,
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
-        set_error("cuTensorMapEncodeTiled failed (CUresult %d) for a KV tensor at %p with %llu rows", (int)r, base,
-                  (unsigned long long)rows);
+        set_error("cuTensorMapEncodeTiled failed (CUresult %d) for a KV tensor at %p with %llu blocks, block stride %llu", (int)r, base,
+                  (unsigned long long)blocks, (unsigned long long)block_stride);
         return EKV_ERR_CUDA;
     }
     return EKV_OK;
@@ -199,7 +200,7 @@ static double now_ms() {
 
 // Undo helper: unmap / release / unreserve whatever a partially built pool holds.
 static void teardown(ekv_pool *p) {
-    const uint64_t layer_bytes = p->base_bytes + p->elastic_bytes;
+    const uint64_t layer_bytes = p->base_bytes + p->elastic_bytes;  // bytes of one range
     for (size_t l = 0; l < p->va.size(); ++l) {
         if (p->grown && p->elastic_held[l]) p->be.unmap(p->be.user, p->va[l] + p->base_bytes, p->elastic_bytes);
         if (p->elastic_held[l]) p->be.release(p->be.user, p->elastic_handle[l]);
@@ -217,7 +218,7 @@ static void teardown(ekv_pool *p) {
 // Map (creating where not held) the elastic handle of every layer.  On failure everything this
 // call mapped or created is undone.
 static ekv_status_t map_elastic(ekv_pool *p) {
-    const int L = p->desc.num_layers;
+    const int L = p->num_ranges;
     std::vector<char> created(L, 0), mapped(L, 0);
     ekv_status_t st = EKV_OK;
     for (int l = 0; l < L && st == EKV_OK; ++l) {
@@ -303,7 +304,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
     if (d.num_layers < 1 || d.num_kv_heads < 1 || d.num_q_heads < d.num_kv_heads || d.num_q_heads % d.num_kv_heads != 0 ||
         d.num_q_heads / d.num_kv_heads > 8 || (d.head_dim != 64 && d.head_dim != 128) || d.block_size != 16 ||
         d.dtype != EKV_BF16 || d.base_blocks < 1 || d.elastic_blocks < 0 || d.device < 0 ||
-        (d.flags & ~(uint32_t)EKV_START_GROWN) != 0) {
+        (d.flags & ~(uint32_t)(EKV_START_GROWN | EKV_FUSED_RANGE)) != 0) {
         set_error("ekv_pool_create: unsupported geometry (layers %d, heads %d/%d, head_dim %d, block_size %d, dtype %d, "
                   "blocks %lld+%lld, flags 0x%x)",
                   d.num_layers, d.num_q_heads, d.num_kv_heads, d.head_dim, d.block_size, d.dtype, (long long)d.base_blocks,
@@ -359,20 +360,26 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
         return EKV_ERR_INVALID;
     }
     p->granularity = gran;
-    p->base_bytes = round_up((uint64_t)d.base_blocks * p->block_bytes, gran);
-    p->elastic_bytes = round_up((uint64_t)d.elastic_blocks * p->block_bytes, gran);
-    p->base_blocks = (int64_t)(p->base_bytes / p->block_bytes);
-    p->elastic_blocks = (int64_t)(p->elastic_bytes / p->block_bytes);
-    const uint64_t layer_bytes = p->base_bytes + p->elastic_bytes;
-    const uint64_t rows = (uint64_t)(p->base_blocks + p->elastic_blocks) * 2ull * d.num_kv_heads * d.block_size;
-    if (rows >= (1ull << 31)) {
-        set_error("ekv_pool_create: %llu KV rows per layer exceed the 2^31 addressing limit", (unsigned long long)rows);
+    p->fused = (d.flags & EKV_FUSED_RANGE) != 0;
+    p->num_ranges = p->fused ? 1 : d.num_layers;
+    const uint64_t per_block = p->fused ? (uint64_t)d.num_layers * p->block_bytes : p->block_bytes;  // range bytes per block id
+    p->block_stride = per_block;
+    // round the block counts UP until a range's base part and elastic part are whole granules
+    uint64_t step = gran / std::__gcd((uint64_t)gran, per_block);  // block counts must be multiples of this
+    p->base_blocks = (int64_t)round_up((uint64_t)d.base_blocks, step);
+    p->elastic_blocks = (int64_t)round_up((uint64_t)d.elastic_blocks, step);
+    p->base_bytes = (uint64_t)p->base_blocks * per_block;
+    p->elastic_bytes = (uint64_t)p->elastic_blocks * per_block;
+    const uint64_t layer_bytes = p->base_bytes + p->elastic_bytes;  // bytes of one range
+    if ((uint64_t)(p->base_blocks + p->elastic_blocks) >= (1ull << 31)) {
+        set_error("ekv_pool_create: %lld block ids per layer exceed the 2^31 addressing limit",
+                  (long long)(p->base_blocks + p->elastic_blocks));
         delete p;
         return EKV_ERR_INVALID;
     }
 
     ekv_status_t st = EKV_OK;
-    for (int l = 0; l < d.num_layers && st == EKV_OK; ++l) {
+    for (int l = 0; l < p->num_ranges && st == EKV_OK; ++l) {
         uint64_t va = 0;
         st = be_status(be.reserve(be.user, layer_bytes, gran, &va), "reserve virtual range", l);
         if (st != EKV_OK) break;
@@ -409,14 +416,18 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
             e = cudaMemcpy(p->d_live, &live, sizeof live, cudaMemcpyHostToDevice);
         }
         if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_layer_base, sizeof(unsigned long long) * d.num_layers);
-        if (e == cudaSuccess)
-            e = cudaMemcpy(p->d_layer_base, p->va.data(), sizeof(unsigned long long) * d.num_layers, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) {
+            std::vector<unsigned long long> bases(d.num_layers);
+            for (int l = 0; l < d.num_layers; ++l) bases[l] = p->layer_base(l);
+            e = cudaMemcpy(p->d_layer_base, bases.data(), sizeof(unsigned long long) * d.num_layers, cudaMemcpyHostToDevice);
+        }
         if (e != cudaSuccess) st = cuda_fail(e, "ekv_pool_create: device state");
-        // One tensor map per layer over the WHOLE range (base + elastic).  Encoding reads no memory,
+        // One tensor map per layer over ALL its block ids (base + elastic).  Encoding reads no memory,
         // and the map never changes when the elastic slice is mapped or unmapped.
         for (int l = 0; l < d.num_layers && st == EKV_OK; ++l) {
             CUtensorMap m;
-            st = encode_kv_map((void *)p->va[l], rows, d.head_dim, d.block_size, &m);
+            st = encode_kv_map((void *)p->layer_base(l), (uint64_t)(p->base_blocks + p->elastic_blocks), p->block_stride,
+                               d.num_kv_heads, d.head_dim, d.block_size, &m);
             if (st != EKV_OK) break;
             p->kv_map.push_back(m);
         }
@@ -459,8 +470,10 @@ ekv_status_t ekv_pool_info(const ekv_pool_t *pool, ekv_pool_info_t *info) {
     memset(info, 0, sizeof *info);
     info->granularity = pool->granularity;
     info->block_bytes = pool->block_bytes;
-    info->base_bytes = pool->base_bytes;
-    info->elastic_bytes = pool->elastic_bytes;
+    info->base_bytes = (uint64_t)pool->base_blocks * pool->block_bytes;        // per layer
+    info->elastic_bytes = (uint64_t)pool->elastic_blocks * pool->block_bytes;  // per layer
+    info->block_stride_bytes = pool->block_stride;
+    info->num_ranges = pool->num_ranges;
     info->base_blocks = pool->base_blocks;
     info->elastic_blocks = pool->elastic_blocks;
     info->live_blocks = pool->base_blocks + (pool->grown ? pool->elastic_blocks : 0);
@@ -477,7 +490,7 @@ ekv_status_t ekv_layer_ptr(const ekv_pool_t *pool, int32_t layer, void **dptr) {
         set_error("ekv_layer_ptr: bad argument");
         return EKV_ERR_INVALID;
     }
-    *dptr = (void *)pool->va[layer];
+    *dptr = (void *)pool->layer_base(layer);
     return EKV_OK;
 }
 
@@ -534,7 +547,7 @@ ekv_status_t ekv_shrink(ekv_pool_t *pool, void *stream, uint32_t flags, double *
     }
     const double t1 = now_ms();
     ekv_status_t st = EKV_OK;
-    for (int l = 0; l < pool->desc.num_layers; ++l) {
+    for (int l = 0; l < pool->num_ranges; ++l) {
         ekv_status_t s1 = be_status(pool->be.unmap(pool->be.user, pool->va[l] + pool->base_bytes, pool->elastic_bytes),
                                     "unmap elastic range", l);
         if (s1 != EKV_OK && st == EKV_OK) st = s1;

@@ -118,12 +118,12 @@ __global__ void __launch_bounds__(128, 2) prefill_mma_kernel(const __grid_consta
         for (int j = 0; j < 4; ++j) {
             int id = ids[(t * 4 + j) % kPmIdCache];
             if (id < 0) id = 0;  // masked below; block 0 is always mapped
-            const int row_k = (id * 2 * p.num_kv_heads + g) * 16;
+            const int row_k = g * 16;  // row inside the block: (K|V, kv-head, token)
             const int row_v = row_k + p.num_kv_heads * 16;
 #pragma unroll
             for (int x = 0; x < BOXES; ++x) {
-                tma_load_2d(dst + j * TILE_BYTES + x * 2048, &kvmap, 64 * x, row_k, bar);
-                tma_load_2d(dst + KV_BYTES + j * TILE_BYTES + x * 2048, &kvmap, 64 * x, row_v, bar);
+                tma_load_3d(dst + j * TILE_BYTES + x * 2048, &kvmap, 64 * x, row_k, id, bar);
+                tma_load_3d(dst + KV_BYTES + j * TILE_BYTES + x * 2048, &kvmap, 64 * x, row_v, id, bar);
             }
         }
     };

@@ -305,7 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             // box b of a tile: block b/2, channel half b%2  ->  [half][block][16 rows][128 B]
             const int b = lane & 15, blk = b >> 1, half = b & 1;
             const int my_id = __shfl_sync(0xffffffffu, id, blk);
-            const int row = (my_id * 2 * p.num_kv_heads + g) * 16 + kv_row_off;
+            const int row = g * 16 + kv_row_off;  // row inside the block: (K|V, kv-head, token)
             if (j >= kStages && !wait_warp(sh, EMPTY + s, (uint32_t)(((j / kStages) - 1) & 1), p.status, p.abort_word)) break;
             if (lane == 0) {
                 if (!is_v) {
@@ -317,7 +317,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             __syncwarp();
             EKV_TRACE(0, j);
             if (lane < 16)
-                tma_load_2d(tile_base + s * kTileBytes + half * kHalfBytes + blk * 2048, &kvmap, 64 * half, row, sh.bar(FULL + s));
+                tma_load_3d(tile_base + s * kTileBytes + half * kHalfBytes + blk * 2048, &kvmap, 64 * half, row, my_id, sh.bar(FULL + s));
             EKV_TRACE(1, j);
         }
     } else if (warp == 1) {

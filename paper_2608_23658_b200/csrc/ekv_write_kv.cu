@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(kWriteThreads) write_kv_kernel(uint4 *__restri
                                                                  const uint4 *__restrict__ v,
                                                                  const long long *__restrict__ slot_mapping, int T,
                                                                  int num_kv_heads, int block_size, int pieces_per_row,
+                                                                 long long block_stride_pieces,
                                                                  const long long *__restrict__ live_ptr, unsigned *status) {
     const long long live = *live_ptr;
     const int row_pieces = num_kv_heads * pieces_per_row;  // one token's K (or V) over all heads
@@ -44,7 +45,7 @@ __global__ void __launch_bounds__(kWriteThreads) write_kv_kernel(uint4 *__restri
                 continue;
             }
             val[u] = (kv ? v : k)[(long long)i * row_pieces + hp];
-            dst[u] = ((((n * 2 + kv) * num_kv_heads + h) * block_size + t) * (long long)pieces_per_row) + c;
+            dst[u] = n * block_stride_pieces + (((long long)(kv * num_kv_heads + h) * block_size + t) * pieces_per_row) + c;
         }
 #pragma unroll
         for (int u = 0; u < kWriteUnroll; ++u)
@@ -71,8 +72,9 @@ extern "C" ekv_status_t ekv_write_kv(ekv_pool_t *pool, int32_t layer, const void
     const long long cap = (long long)pool->sm_count * 8;  // 8 CTAs of 256 threads per SM: one full wave
     if (blocks > cap) blocks = cap;
     write_kv_kernel<<<(unsigned)blocks, kWriteThreads, 0, (cudaStream_t)stream>>>(
-        (uint4 *)pool->va[layer], (const uint4 *)k, (const uint4 *)v, (const long long *)slot_mapping, T,
-        pool->desc.num_kv_heads, pool->desc.block_size, pieces_per_row, pool->d_live, pool->d_status);
+        (uint4 *)pool->layer_base(layer), (const uint4 *)k, (const uint4 *)v, (const long long *)slot_mapping, T,
+        pool->desc.num_kv_heads, pool->desc.block_size, pieces_per_row, (long long)(pool->block_stride / 16), pool->d_live,
+        pool->d_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_write_kv launch");
     return EKV_OK;

@@ -17,13 +17,13 @@ class _RawCuda:
 
 class Pool:
     def __init__(self, *, num_q_heads, num_kv_heads, head_dim, base_blocks, elastic_blocks=0, num_layers=1,
-                 block_size=16, device=0, start_grown=False):
+                 block_size=16, device=0, start_grown=False, fused_range=False):
         self.device = torch.device("cuda", device)
         torch.cuda.set_device(self.device)
         self.handle = B.ekv_pool_create(device=device, num_layers=num_layers, num_q_heads=num_q_heads,
                                         num_kv_heads=num_kv_heads, head_dim=head_dim, block_size=block_size,
                                         base_blocks=base_blocks, elastic_blocks=elastic_blocks,
-                                        flags=B.EKV_START_GROWN if start_grown else 0)
+                                        flags=(B.EKV_START_GROWN if start_grown else 0) | (B.EKV_FUSED_RANGE if fused_range else 0))
         self.num_q_heads, self.num_kv_heads, self.head_dim, self.block_size = num_q_heads, num_kv_heads, head_dim, block_size
         self.num_layers = num_layers
         self._ws = None
@@ -65,9 +65,13 @@ class Pool:
         if first_block < 0 or first_block + num_blocks > info.live_blocks:
             raise ValueError("view would reach past the live (mapped) blocks")
         elems = info.block_bytes // 2
-        raw = _RawCuda(self.layer_ptr(layer) + first_block * info.block_bytes, num_blocks * elems)
-        t = torch.as_tensor(raw, device=self.device).view(torch.bfloat16)
-        return t.view(num_blocks, 2, self.num_kv_heads, self.block_size, self.head_dim)
+        stride = info.block_stride_bytes // 2      # elements between consecutive block ids of this layer
+        span = (num_blocks - 1) * stride + elems if num_blocks > 0 else 0
+        raw = _RawCuda(self.layer_ptr(layer) + first_block * info.block_stride_bytes, max(span, 1))
+        flat = torch.as_tensor(raw, device=self.device).view(torch.bfloat16)
+        d, bs, hk = self.head_dim, self.block_size, self.num_kv_heads
+        # dense when stride == elems (one range per layer); a strided view over the fused range otherwise
+        return torch.as_strided(flat, (num_blocks, 2, hk, bs, d), (stride, hk * bs * d, bs * d, d, 1))
 
     def grow(self, stream=None):
         return B.ekv_grow(self.handle, stream)
