@@ -174,3 +174,29 @@ def test_argument_checks_and_host_only_refusal(vmm):
         ekv.ekv_set_vmm_backend(None)                           # pools still exist
     assert e.value.status == ekv.Status.ERR_STATE
     ekv.ekv_pool_destroy(pool)
+
+
+def test_fused_range_is_one_reservation_and_two_handles_for_all_layers(vmm):
+    # 3 layers x 64 KiB blocks: a block id spans 192 KiB of the range, so counts round up to multiples of 32
+    pool = _create(num_layers=3, base_blocks=100, elastic_blocks=40, flags=ekv.EKV_FUSED_RANGE)
+    info = ekv.ekv_pool_info(pool)
+    assert (info.base_blocks, info.elastic_blocks) == (128, 64)
+    assert info.num_ranges == 1 and info.block_stride_bytes == 3 * 64 * 1024 and info.block_bytes == 64 * 1024
+    assert len(vmm.reserved) == 1 and len(vmm.handles) == 1 and len(vmm.mapped) == 1
+    (va, size), = vmm.reserved.items()
+    assert size == (128 + 64) * 3 * 64 * 1024
+    assert [ekv.ekv_layer_ptr(pool, l) for l in range(3)] == [va + l * 64 * 1024 for l in range(3)]
+    n_calls = len(vmm.log)
+    ekv.ekv_grow(pool, host_only=True)
+    assert [e[0] for e in vmm.log[n_calls:]] == ["create", "map"]       # one create + one map for the whole model
+    assert vmm.mapped[va + 128 * 3 * 64 * 1024][0] == 64 * 3 * 64 * 1024  # the elastic ids are the top of the range
+    assert ekv.ekv_pool_info(pool).live_blocks == 192
+    n_calls = len(vmm.log)
+    ekv.ekv_shrink(pool, host_only=True)
+    assert [e[0] for e in vmm.log[n_calls:]] == ["unmap", "release"]
+    vmm.fail_map_at = 0
+    with pytest.raises(ekv.EkvError):
+        ekv.ekv_grow(pool, host_only=True)
+    assert len(vmm.handles) == 1 and len(vmm.mapped) == 1 and not ekv.ekv_pool_info(pool).grown
+    ekv.ekv_pool_destroy(pool)
+    assert not vmm.reserved and not vmm.handles and not vmm.mapped
