@@ -303,14 +303,14 @@ def measure_prefill(device, peaks, reps=3, prompt_len=None, chunks=None):
         pool.close()
 
 
-def _toggle_modes(device, num_layers, per_layer_bytes, cycles):
+def _toggle_modes(device, num_layers, per_layer_bytes, cycles, fused=False):
     """grow / shrink ms for one geometry, three ways: keep the range and re-create the handle (default), keep
     range and handle (EKV_KEEP_PHYSICAL), and the naive way -- a fresh range + handle + mapping per toggle."""
     import paper_2608_23658_b200 as ekv
     s = I.C5.shape
     el_blocks = per_layer_bytes // s.block_bytes
     geom = dict(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, num_layers=num_layers,
-                device=device.index or 0)
+                device=device.index or 0, fused_range=fused)
     pool = ekv.Pool(base_blocks=el_blocks + 512, elastic_blocks=el_blocks, **geom)
     try:
         rows = {"grow_release": [], "shrink_release": [], "grow_keep": [], "shrink_keep": []}
@@ -360,6 +360,8 @@ def measure_toggle(device, cycles=5):
     microbenchmark geometry (28 layers, 3.09 GiB in all; its numbers are from another machine: context only)."""
     cfg = I.C5
     out = _toggle_modes(device, cfg.num_layers, cfg.elastic_total_bytes // cfg.num_layers, cycles)
+    # the same reserve as ONE range and two handles for all layers (EKV_FUSED_RANGE): one map / unmap per toggle
+    out["fused_range"] = _toggle_modes(device, cfg.num_layers, cfg.elastic_total_bytes // cfg.num_layers, cycles, fused=True)
     out["paper_geometry_28_layers"] = _toggle_modes(device, 28, (int(3.09 * 2**30) // 28 // (2 << 20) + 1) * (2 << 20), cycles)
     out["paper_a100_context_ms"] = {"decommit": 3.0, "commit": 30.0, "naive_commit": 180.0, "live_decommit": 3.8, "live_commit": 23.8}
     return out
