@@ -222,9 +222,18 @@ KV_STREAM = 21  # stream id of "pool content as a function of the physical eleme
 
 def fill_pool_layer_(layer_view: torch.Tensor, seed: int, layer: int = 0, first_block: int = 0, chunk: int = 1 << 24) -> None:
     """Fill a [blocks, 2, Hkv, bs, d] bf16 view of a layer (starting at physical block first_block)
-    so that element e of the layer holds normal_bf16(seed, KV_STREAM + layer, e)."""
+    so that element e of the layer holds normal_bf16(seed, KV_STREAM + layer, e).  The view may be strided
+    between blocks (a layer of a fused range); each block itself is dense."""
     block_elems = layer_view[0].numel()
-    fill_normal_bf16_(layer_view, seed, KV_STREAM + layer, start=first_block * block_elems, chunk=chunk)
+    if layer_view.is_contiguous():
+        fill_normal_bf16_(layer_view, seed, KV_STREAM + layer, start=first_block * block_elems, chunk=chunk)
+        return
+    per = max(1, chunk // block_elems)
+    for b0 in range(0, layer_view.shape[0], per):
+        b1 = min(layer_view.shape[0], b0 + per)
+        vals = normal_bf16(seed, KV_STREAM + layer, (first_block + b0) * block_elems, (b1 - b0) * block_elems,
+                           device=layer_view.device)
+        layer_view[b0:b1] = vals.view(b1 - b0, *layer_view.shape[1:])
 
 
 def host_blocks(seed: int, layer: int, block_ids, block_elems: int) -> torch.Tensor:

@@ -184,12 +184,14 @@ def test_c4_long_context_70b_shape_with_elastic_blocks():
 # ------------------------------------------------------------------ configs[4]
 
 
-def test_c5_elastic_toggle_under_load():
+@pytest.mark.parametrize("fused", [False, True])
+def test_c5_elastic_toggle_under_load(fused):
     """32 layers, batch 128, 1000 decode steps (EKV_C5_STEPS overrides), shrink/grow alternating every 50 steps.
+    fused=True repeats the protocol (300 steps) on a pool with ONE range for all layers (EKV_FUSED_RANGE).
     112 tenants live in base blocks only; 16 'straddlers' take their new blocks from the elastic range while it
     is mapped and are drained to spare base blocks before every shrink."""
     cfg, s = I.C5, I.C5.shape
-    steps = int(os.environ.get("EKV_C5_STEPS", cfg.steps))
+    steps = int(os.environ.get("EKV_C5_STEPS", 300 if fused else cfg.steps))
     NL, B, every = cfg.num_layers, cfg.decode.batch, cfg.toggle_every
     lengths = I.decode_lengths(cfg)
     elastic_blocks = cfg.elastic_total_bytes // NL // s.block_bytes
@@ -199,9 +201,10 @@ def test_c5_elastic_toggle_under_load():
     free, _ = torch.cuda.mem_get_info()
     assert need_bytes + 3 * GiB < free, f"configs[4] needs {need_bytes / GiB:.1f} GiB, device has {free / GiB:.1f} GiB free"
     pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=base_blocks,
-                    elastic_blocks=elastic_blocks, num_layers=NL, start_grown=True)
+                    elastic_blocks=elastic_blocks, num_layers=NL, start_grown=True, fused_range=fused)
     try:
         info = pool.info
+        assert info.num_ranges == (1 if fused else NL)
         base, el = info.base_blocks, info.elastic_blocks
         for l in range(NL):
             I.fill_pool_layer_(pool.layer_tensor(l, 0, base), cfg.seed, layer=l)
@@ -305,7 +308,7 @@ def test_c5_elastic_toggle_under_load():
                                   torch.arange(nb, dtype=torch.int32)[None], np.array([L1]), scale)
         check_close(last, want, "C5 sampled tenant after all steps")
         ms = {k: [round(t[0], 2) for t in v] for k, v in toggles.items()}
-        print(f"\nC5 toggles (driver-call ms; the whole call also drains the queued steps), {NL} layers x "
+        print(f"\nC5 toggles{' (fused range)' if fused else ''} (driver-call ms; the whole call also drains the queued steps), {NL} layers x "
               f"{el * s.block_bytes >> 20} MiB: {ms}")
     finally:
         pool.close()
