@@ -7,7 +7,7 @@
 //
 //   warp 0        TMA producer: 16-token x 64-channel boxes (128-byte swizzle) of K and V blocks,
 //                 gathered through the block table into 128-key tiles, 2 stages each for K and V
-//   warp 1        MMA issuer (one thread): S = Q K^T (A, B from shared memory, K-major) and
+//   warp 1        MMA issuer (whole warp converged, one elected lane issues): S = Q K^T (A, B from shared memory, K-major) and
 //                 O += P V (A = P read from TMEM, B = V from shared memory, MN-major)
 //   warp 2        TMEM allocation / release (512 columns: S_A S_B O_A O_B, P aliases S)
 //   warps 4-7     softmax of head A: one thread per query row (= TMEM lane)
@@ -74,25 +74,31 @@ static constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
     return ((addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
 }
+// These three are executed by the WHOLE (converged) issuing warp with warp-uniform operands; one lane, picked by
+// elect.sync inside the block, issues the instruction.  Written this way the operands can live in uniform
+// registers; wrapped in `if (lane == 0)` they are per-thread values that have to be moved over one by one.
 template <bool kAcc>
 __device__ __forceinline__ void mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %5, 0;\n\t"
         "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHi), "r"(idesc), "n"(kAcc ? 1 : 0)
         : "memory");
 }
 __device__ __forceinline__ void mma_ts_lo_dyn(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "{\n\t.reg .pred p, e;\n\t.reg .b64 db;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %5, 0;\n\t"
         "mov.b64 db, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHi), "r"(idesc), "r"(acc)
         : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+        "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar)
+        : "memory");
 }
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -317,14 +323,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         EKV_TRACE(7, 0);
         if (ok) {
             fence_after();
-            if (lane == 0) {
-                issue_qk(0, 0);
-                mma_commit(sh.bar(S_READY + 0));
-                issue_qk(1, 0);
-                mma_commit(sh.bar(K_EMPTY + 0));
-                mma_commit(sh.bar(S_READY + 1));
-            }
-            __syncwarp();
+            issue_qk(0, 0);
+            mma_commit(sh.bar(S_READY + 0));
+            issue_qk(1, 0);
+            mma_commit(sh.bar(K_EMPTY + 0));
+            mma_commit(sh.bar(S_READY + 1));
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const int s = j % kStages, s1 = (j + 1) % kStages;
                 const bool more = j + 1 < n_tiles;
@@ -334,43 +337,34 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 if (ok) ok = wait_warp(sh, P_PART + 0, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
                 fence_after();
-                if (lane == 0) issue_pv(0, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
-                __syncwarp();
+                issue_pv(0, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
                 ok = wait_warp(sh, P_READY + 0, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
                 EKV_TRACE(1, j);
                 fence_after();
-                if (lane == 0) {
-                    issue_pv(0, s, true, kPartSteps, kBN / 16);
-                    if (more) issue_qk(0, s1);
-                    mma_commit(sh.bar(S_READY + 0));
-                }
-                __syncwarp();
+                issue_pv(0, s, true, kPartSteps, kBN / 16);
+                if (more) issue_qk(0, s1);
+                mma_commit(sh.bar(S_READY + 0));
                 EKV_TRACE(2, j);
                 ok = wait_warp(sh, P_PART + 1, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
                 fence_after();
-                if (lane == 0) issue_pv(1, s, j > 0, 0, kPartSteps);
-                __syncwarp();
+                issue_pv(1, s, j > 0, 0, kPartSteps);
                 ok = wait_warp(sh, P_READY + 1, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
                 EKV_TRACE(3, j);
                 fence_after();
-                if (lane == 0) {
-                    issue_pv(1, s, true, kPartSteps, kBN / 16);
-                    mma_commit(sh.bar(V_EMPTY + s));
-                    if (more) {
-                        issue_qk(1, s1);
-                        mma_commit(sh.bar(K_EMPTY + s1));
-                    }
-                    mma_commit(sh.bar(S_READY + 1));
+                issue_pv(1, s, true, kPartSteps, kBN / 16);
+                mma_commit(sh.bar(V_EMPTY + s));
+                if (more) {
+                    issue_qk(1, s1);
+                    mma_commit(sh.bar(K_EMPTY + s1));
                 }
-                __syncwarp();
+                mma_commit(sh.bar(S_READY + 1));
             }
         }
         // every MMA this thread issued must be finished before TMEM is released
-        if (lane == 0) mma_commit(sh.bar(DRAIN));
-        __syncwarp();
+        mma_commit(sh.bar(DRAIN));
         (void)wait_warp(sh, DRAIN, 0, p.status, p.abort_word);
     }
     } else {
