@@ -303,6 +303,79 @@ def measure_prefill(device, peaks, reps=3, prompt_len=None, chunks=None):
         pool.close()
 
 
+def measure_mixed_step(device, peaks, reps=5):
+    """configs[2] as one engine step: the last 8192-token chunk of the 32768-token prompt (cached prefix 24576)
+    co-scheduled with the 256-sequence decode batch.  Timed three ways: each call alone, both back to back on
+    one stream, and both at once on two streams (what a scheduler that batches them gets)."""
+    import paper_2608_23658_b200 as ekv
+    cfg, s = I.C3, I.C3.shape
+    Lp, chunk = cfg.prompt_len, 8192
+    lengths = torch.cat([torch.tensor([Lp]), I.decode_lengths(cfg)])
+    need = int(I.blocks_for(lengths, s.block_size).sum())
+    pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim,
+                    base_blocks=int(need * 1.05) + 64, device=device.index or 0)
+    try:
+        tables, _ = I.assign_blocks(cfg.seed, 14, lengths, s.block_size, pool.info.live_blocks)
+        I.fill_pool_layer_(pool.layer_tensor(0), cfg.seed)
+        B = len(lengths) - 1
+        d_tables = tables.to(device)
+        p_table, d_table = d_tables[:1].contiguous(), d_tables[1:].contiguous()
+        d_lens = lengths[1:].to(torch.int32).to(device)
+        qp = I.normal_bf16(cfg.seed, 6, 0, chunk * s.num_q_heads * s.head_dim, device=device).view(chunk, s.num_q_heads, s.head_dim)
+        qd = I.normal_bf16(cfg.seed, 7, 0, B * s.num_q_heads * s.head_dim, device=device).view(B, s.num_q_heads, s.head_dim)
+        op, od = torch.empty_like(qp), torch.empty_like(qd)
+        cu_h = torch.tensor([0, chunk], dtype=torch.int32)
+        cu_d = cu_h.to(device)
+        p_len = torch.tensor([Lp], dtype=torch.int32, device=device)
+        ws = pool.workspace(B, int(d_table.shape[1]) * s.block_size)
+        scale = 1.0 / math.sqrt(s.head_dim)
+        side = torch.cuda.Stream(device)
+        main = torch.cuda.current_stream(device)
+
+        def prefill():
+            pool.attn_prefill_chunk(0, qp, p_table, cu_d, cu_h, p_len, scale, out=op)
+
+        def decode():
+            pool.attn_decode(0, qd, d_table, d_lens, scale, out=od, workspace=ws)
+
+        def serial():
+            prefill()
+            decode()
+
+        def concurrent():
+            fork, join = torch.cuda.Event(), torch.cuda.Event()
+            fork.record(main)
+            side.wait_event(fork)
+            with torch.cuda.stream(side):
+                decode()
+                join.record(side)
+            prefill()
+            main.wait_event(join)
+
+        def best_of(fn):
+            fn()
+            torch.cuda.synchronize(device)
+            best = float("inf")
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize(device)
+                best = min(best, e0.elapsed_time(e1))
+            return best
+
+        t_p, t_d, t_s, t_c = best_of(prefill), best_of(decode), best_of(serial), best_of(concurrent)
+        flops = I.prefill_flops(chunk, Lp - chunk, s)
+        dbytes = I.decode_algorithmic_bytes(lengths[1:], s)
+        return {"prefill_alone_ms": round(t_p, 3), "prefill_alone_tflops": round(flops / (t_p * 1e-3) / 1e12, 1),
+                "decode_alone_ms": round(t_d, 3), "decode_alone_gbs": round(dbytes / (t_d * 1e-3) / 1e9, 1),
+                "serial_ms": round(t_s, 3), "two_streams_ms": round(t_c, 3),
+                "workload": "c3 step: 8192-token chunk over a 24576-token cached prefix + 256 decode sequences U[2048,8192]"}
+    finally:
+        pool.close()
+
+
 def _toggle_modes(device, num_layers, per_layer_bytes, cycles, fused=False):
     """grow / shrink ms for one geometry, three ways: keep the range and re-create the handle (default), keep
     range and handle (EKV_KEEP_PHYSICAL), and the naive way -- a fresh range + handle + mapping per toggle."""
@@ -604,6 +677,8 @@ def main():
     if rank == 0 and world == 1 and not args.no_extras:
         torch.cuda.empty_cache()
         line["prefill"] = measure_prefill(device, peaks)
+        torch.cuda.empty_cache()
+        line["mixed_step"] = measure_mixed_step(device, peaks)
         torch.cuda.empty_cache()
         line["toggle"] = measure_toggle(device)
         torch.cuda.empty_cache()

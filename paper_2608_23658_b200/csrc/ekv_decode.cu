@@ -417,6 +417,47 @@ static ekv_status_t launch_decode(ekv_pool *pool, int layer, const DecodeParams 
     return launch_decode_impl<D, false>(pool, pool->kv_map[layer], pool->kv_map[layer], p, B, stream);
 }
 
+
+// Argument checks shared by the three decode entry points.
+static ekv_status_t check_decode_args(const char *who, const void *q, const void *out, const int32_t *block_tables,
+                                      int32_t max_blocks_per_seq, const int32_t *seq_lens, int32_t B) {
+    if (B < 0 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26) || B > 65535 ||
+        (B > 0 && (!q || !out || !block_tables || !seq_lens)) || ((uintptr_t)q & 15) || ((uintptr_t)out & 15)) {
+        set_error("%s: bad argument (B=%d, max_blocks_per_seq=%d)", who, B, max_blocks_per_seq);
+        return EKV_ERR_INVALID;
+    }
+    return EKV_OK;
+}
+
+// Kernel parameters of one call; `scratch` holds the (m, l) pairs first, then the partial rows.
+static DecodeParams make_decode_params(const ekv_pool *pool, const DecodePlan &plan, const void *q, void *out,
+                                       const int32_t *block_tables, int32_t max_blocks_per_seq, const int32_t *seq_lens, int32_t B,
+                                       float scale, void *scratch) {
+    const size_t parts = (size_t)B * pool->desc.num_q_heads * plan.nsplit;
+    DecodeParams p;
+    p.q = (const __nv_bfloat16 *)q;
+    p.block_tables = block_tables;
+    p.seq_lens = seq_lens;
+    p.live = pool->d_live;
+    p.status = pool->d_status;
+    p.part_ml = (float2 *)scratch;
+    p.part_o = (float *)((uint8_t *)scratch + (parts * sizeof(float2) + 255) / 256 * 256);
+    p.out = (__nv_bfloat16 *)out;
+    p.max_blocks = max_blocks_per_seq;
+    p.num_q_heads = pool->desc.num_q_heads;
+    p.num_kv_heads = pool->desc.num_kv_heads;
+    p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
+    p.chunk_tokens = plan.chunk_tokens;
+    p.nsplit = plan.nsplit;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.first_tensor_blocks = p.total_blocks = 0;
+    return p;
+}
+
+static ekv_status_t dispatch_decode(ekv_pool *pool, int layer, const DecodeParams &p, int B, cudaStream_t stream) {
+    if (pool->desc.head_dim == 128) return launch_decode<128>(pool, layer, p, B, stream);
+    return launch_decode<64>(pool, layer, p, B, stream);
+}
 }  // namespace ekv
 
 using namespace ekv;
@@ -437,12 +478,8 @@ extern "C" ekv_status_t ekv_attn_decode(ekv_pool_t *pool, int32_t layer, const v
                                         const int32_t *block_tables, int32_t max_blocks_per_seq, const int32_t *seq_lens,
                                         int32_t B, float scale, void *workspace, size_t workspace_bytes, void *stream) {
     ekv_status_t st = check_compute(pool, layer, "ekv_attn_decode");
+    if (st == EKV_OK) st = check_decode_args("ekv_attn_decode", q, out, block_tables, max_blocks_per_seq, seq_lens, B);
     if (st != EKV_OK) return st;
-    if (B < 0 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26) || B > 65535 ||
-        (B > 0 && (!q || !out || !block_tables || !seq_lens)) || ((uintptr_t)q & 15) || ((uintptr_t)out & 15)) {
-        set_error("ekv_attn_decode: bad argument (B=%d, max_blocks_per_seq=%d)", B, max_blocks_per_seq);
-        return EKV_ERR_INVALID;
-    }
     if (B == 0) return EKV_OK;
     const DecodePlan plan = plan_decode(pool, B, max_blocks_per_seq);
     const size_t need = decode_workspace_need(pool, B, plan.nsplit);
@@ -451,26 +488,8 @@ extern "C" ekv_status_t ekv_attn_decode(ekv_pool_t *pool, int32_t layer, const v
                   need);
         return EKV_ERR_WORKSPACE;
     }
-    const size_t parts = (size_t)B * pool->desc.num_q_heads * plan.nsplit;
-    DecodeParams p;
-    p.q = (const __nv_bfloat16 *)q;
-    p.block_tables = block_tables;
-    p.seq_lens = seq_lens;
-    p.live = pool->d_live;
-    p.status = pool->d_status;
-    p.part_ml = (float2 *)workspace;
-    p.part_o = (float *)((uint8_t *)workspace + (parts * sizeof(float2) + 255) / 256 * 256);
-    p.out = (__nv_bfloat16 *)out;
-    p.max_blocks = max_blocks_per_seq;
-    p.num_q_heads = pool->desc.num_q_heads;
-    p.num_kv_heads = pool->desc.num_kv_heads;
-    p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
-    p.chunk_tokens = plan.chunk_tokens;
-    p.nsplit = plan.nsplit;
-    p.scale_log2 = scale * 1.4426950408889634f;
-    p.first_tensor_blocks = p.total_blocks = 0;
-    if (pool->desc.head_dim == 128) return launch_decode<128>(pool, layer, p, B, (cudaStream_t)stream);
-    return launch_decode<64>(pool, layer, p, B, (cudaStream_t)stream);
+    const DecodeParams p = make_decode_params(pool, plan, q, out, block_tables, max_blocks_per_seq, seq_lens, B, scale, workspace);
+    return dispatch_decode(pool, layer, p, B, (cudaStream_t)stream);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -516,12 +535,8 @@ extern "C" ekv_status_t ekv_attn_decode_static_scratch(ekv_pool_t *pool, int32_t
                                                        const int32_t *block_tables, int32_t max_blocks_per_seq,
                                                        const int32_t *seq_lens, int32_t B, float scale, void *stream) {
     ekv_status_t st = check_compute(pool, layer, "ekv_attn_decode_static_scratch");  // makes the pool's device current
+    if (st == EKV_OK) st = check_decode_args("ekv_attn_decode_static_scratch", q, out, block_tables, max_blocks_per_seq, seq_lens, B);
     if (st != EKV_OK) return st;
-    if (B < 0 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26) || B > 65535 ||
-        (B > 0 && (!q || !out || !block_tables || !seq_lens)) || ((uintptr_t)q & 15) || ((uintptr_t)out & 15)) {
-        set_error("ekv_attn_decode_static_scratch: bad argument (B=%d, max_blocks_per_seq=%d)", B, max_blocks_per_seq);
-        return EKV_ERR_INVALID;
-    }
     if (B == 0) return EKV_OK;
     const DecodePlan plan = plan_decode(pool, B, max_blocks_per_seq);
     const size_t need = decode_workspace_need(pool, B, plan.nsplit);
@@ -534,28 +549,9 @@ extern "C" ekv_status_t ekv_attn_decode_static_scratch(ekv_pool_t *pool, int32_t
     void *scratch = nullptr;
     st = static_scratch_address(pool->desc.device, &scratch);
     if (st != EKV_OK) return st;
-    const size_t parts = (size_t)B * pool->desc.num_q_heads * plan.nsplit;
-    DecodeParams p;
-    p.q = (const __nv_bfloat16 *)q;
-    p.block_tables = block_tables;
-    p.seq_lens = seq_lens;
-    p.live = pool->d_live;
-    p.status = pool->d_status;
-    p.part_ml = (float2 *)scratch;
-    p.part_o = (float *)((uint8_t *)scratch + (parts * sizeof(float2) + 255) / 256 * 256);
-    p.out = (__nv_bfloat16 *)out;
-    p.max_blocks = max_blocks_per_seq;
-    p.num_q_heads = pool->desc.num_q_heads;
-    p.num_kv_heads = pool->desc.num_kv_heads;
-    p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
-    p.chunk_tokens = plan.chunk_tokens;
-    p.nsplit = plan.nsplit;
-    p.scale_log2 = scale * 1.4426950408889634f;
-    p.first_tensor_blocks = p.total_blocks = 0;
-    if (pool->desc.head_dim == 128) return launch_decode<128>(pool, layer, p, B, (cudaStream_t)stream);
-    return launch_decode<64>(pool, layer, p, B, (cudaStream_t)stream);
+    const DecodeParams p = make_decode_params(pool, plan, q, out, block_tables, max_blocks_per_seq, seq_lens, B, scale, scratch);
+    return dispatch_decode(pool, layer, p, B, (cudaStream_t)stream);
 }
-
 
 // ------------------------------------------------------------------------------------------------
 // The two-tensor alternative (paper, "The contiguity constraint": split the KV into two tensors and
@@ -568,19 +564,13 @@ extern "C" ekv_status_t ekv_attn_decode_two_tensor(ekv_pool_t *pool, int32_t lay
                                                    int32_t max_blocks_per_seq, const int32_t *seq_lens, int32_t B, float scale,
                                                    void *workspace, size_t workspace_bytes, void *stream) {
     ekv_status_t st = check_compute(pool, layer, "ekv_attn_decode_two_tensor");
+    if (st == EKV_OK) st = check_decode_args("ekv_attn_decode_two_tensor", q, out, block_tables, max_blocks_per_seq, seq_lens, B);
     if (st != EKV_OK) return st;
-    if (B < 0 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26) || B > 65535 || second_blocks < 1 || !second_tensor ||
-        ((uintptr_t)second_tensor & 15) || (B > 0 && (!q || !out || !block_tables || !seq_lens)) || ((uintptr_t)q & 15) ||
-        ((uintptr_t)out & 15)) {
-        set_error("ekv_attn_decode_two_tensor: bad argument (B=%d, max_blocks_per_seq=%d, second_blocks=%lld)", B, max_blocks_per_seq,
-                  (long long)second_blocks);
+    if (second_blocks < 1 || second_blocks >= (1ll << 31) || !second_tensor || ((uintptr_t)second_tensor & 15)) {
+        set_error("ekv_attn_decode_two_tensor: bad second tensor (%p, %lld blocks)", second_tensor, (long long)second_blocks);
         return EKV_ERR_INVALID;
     }
     if (B == 0) return EKV_OK;
-    if (second_blocks >= (1ll << 31)) {
-        set_error("ekv_attn_decode_two_tensor: second tensor too large");
-        return EKV_ERR_INVALID;
-    }
     const DecodePlan plan = plan_decode(pool, B, max_blocks_per_seq);
     const size_t need = decode_workspace_need(pool, B, plan.nsplit);
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) {
@@ -592,23 +582,7 @@ extern "C" ekv_status_t ekv_attn_decode_two_tensor(ekv_pool_t *pool, int32_t lay
     st = encode_kv_map(const_cast<void *>(second_tensor), (uint64_t)second_blocks, pool->block_bytes, pool->desc.num_kv_heads,
                        pool->desc.head_dim, pool->desc.block_size, &map2);
     if (st != EKV_OK) return st;
-    const size_t parts = (size_t)B * pool->desc.num_q_heads * plan.nsplit;
-    DecodeParams p;
-    p.q = (const __nv_bfloat16 *)q;
-    p.block_tables = block_tables;
-    p.seq_lens = seq_lens;
-    p.live = pool->d_live;
-    p.status = pool->d_status;
-    p.part_ml = (float2 *)workspace;
-    p.part_o = (float *)((uint8_t *)workspace + (parts * sizeof(float2) + 255) / 256 * 256);
-    p.out = (__nv_bfloat16 *)out;
-    p.max_blocks = max_blocks_per_seq;
-    p.num_q_heads = pool->desc.num_q_heads;
-    p.num_kv_heads = pool->desc.num_kv_heads;
-    p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
-    p.chunk_tokens = plan.chunk_tokens;
-    p.nsplit = plan.nsplit;
-    p.scale_log2 = scale * 1.4426950408889634f;
+    DecodeParams p = make_decode_params(pool, plan, q, out, block_tables, max_blocks_per_seq, seq_lens, B, scale, workspace);
     p.first_tensor_blocks = pool->base_blocks;  // the first tensor is the pool's base range, whatever the elastic state
     p.total_blocks = pool->base_blocks + second_blocks;
     if (pool->desc.head_dim == 128)

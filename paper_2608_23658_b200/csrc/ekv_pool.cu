@@ -9,6 +9,7 @@
 #include <chrono>
 #include <mutex>
 #include <new>
+#include <numeric>
 
 #include "ekv_internal.h"
 
@@ -365,7 +366,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
     const uint64_t per_block = p->fused ? (uint64_t)d.num_layers * p->block_bytes : p->block_bytes;  // range bytes per block id
     p->block_stride = per_block;
     // round the block counts UP until a range's base part and elastic part are whole granules
-    uint64_t step = gran / std::__gcd((uint64_t)gran, per_block);  // block counts must be multiples of this
+    uint64_t step = gran / std::gcd((uint64_t)gran, per_block);  // block counts must be multiples of this
     p->base_blocks = (int64_t)round_up((uint64_t)d.base_blocks, step);
     p->elastic_blocks = (int64_t)round_up((uint64_t)d.elastic_blocks, step);
     p->base_bytes = (uint64_t)p->base_blocks * per_block;
@@ -573,8 +574,15 @@ ekv_status_t ekv_poll_status(ekv_pool_t *pool) {
     }
     if (pool->host_only) return EKV_OK;
     unsigned v = __atomic_exchange_n(pool->h_status, 0u, __ATOMIC_ACQ_REL);
-    if (v & EKV_DEV_FLAG_TIMEOUT) return EKV_ERR_TIMEOUT;
-    if (v & EKV_DEV_FLAG_OOB) return EKV_ERR_BLOCK_OOB;
+    if (v & EKV_DEV_FLAG_TIMEOUT) {
+        set_error("ekv_poll_status: a kernel gave up a bounded wait since the last poll%s",
+                  (v & EKV_DEV_FLAG_OOB) ? " (and skipped a block id outside the live range)" : "");
+        return EKV_ERR_TIMEOUT;
+    }
+    if (v & EKV_DEV_FLAG_OOB) {
+        set_error("ekv_poll_status: a kernel skipped a block id (or slot) outside the live range since the last poll");
+        return EKV_ERR_BLOCK_OOB;
+    }
     return EKV_OK;
 }
 
