@@ -159,50 +159,24 @@ class DecodeWorkload:
             ev[2].record()
 
     def setup_e2e(self):
-        """Second set of device input / output buffers and the copy streams of the end-to-end pipeline."""
-        dev = self.dev
-        self.s_in, self.s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
-        self.bufs = []
-        for _ in range(2):
-            self.bufs.append({
-                "q": torch.empty_like(self.q), "k": torch.empty_like(self.k), "v": torch.empty_like(self.v),
-                "slots": torch.empty_like(self.slots), "tables": torch.empty_like(self.d_tables),
-                "lens": torch.empty_like(self.d_lens), "out": torch.empty_like(self.out),
-                "h_out": torch.empty_like(self.h_out).pin_memory(),
-                "ev_in": torch.cuda.Event(), "ev_comp": torch.cuda.Event(), "ev_out": torch.cuda.Event()})
+        """The end-to-end pipeline: ekv_hoststep_* with two staging sets (copies on the library's own streams)."""
+        self.hs = self.ekv.HostStep(self.pool, self.B, int(self.tables.shape[1]), depth=2)
+        self.h_outs = [torch.empty_like(self.h_out).pin_memory() for _ in range(2)]
         self.e2e_i = 0
 
     def step_e2e(self):
-        """Same step through host buffers: every step copies its inputs from pinned host memory and its
-        result back to the host.  Copies run on their own streams and are double-buffered, so the H2D of
-        step i+1 and the D2H of step i-1 overlap the kernels of step i; every byte still moves every step."""
-        b = self.bufs[self.e2e_i % 2]
+        """Same step through HOST buffers, one C-ABI call: every step copies its inputs from pinned host memory,
+        runs ekv_write_kv + ekv_attn_decode and copies its result back to the host.  The copies are double-buffered
+        against the kernels (the H2D of step i+1 and the D2H of step i-1 overlap the kernels of step i); every byte
+        still moves every step."""
+        out = self.h_outs[self.e2e_i % 2]
         self.e2e_i += 1
-        main = torch.cuda.current_stream(self.dev)
-        with torch.cuda.stream(self.s_in):
-            self.s_in.wait_event(b["ev_comp"])          # the kernels that last read this buffer set are done
-            b["q"].copy_(self.h_q, non_blocking=True)
-            b["k"].copy_(self.h_k, non_blocking=True)
-            b["v"].copy_(self.h_v, non_blocking=True)
-            b["slots"].copy_(self.h_slots, non_blocking=True)
-            b["tables"].copy_(self.h_tables, non_blocking=True)
-            b["lens"].copy_(self.h_lens, non_blocking=True)
-            b["ev_in"].record(self.s_in)
-        main.wait_event(b["ev_in"])
-        main.wait_event(b["ev_out"])                     # the previous result in this set has left the device
-        self.pool.write_kv(0, b["k"], b["v"], b["slots"])
-        self.pool.attn_decode(0, b["q"], b["tables"], b["lens"], self.scale, out=b["out"], workspace=self.ws)
-        b["ev_comp"].record(main)
-        with torch.cuda.stream(self.s_out):
-            self.s_out.wait_event(b["ev_comp"])
-            b["h_out"].copy_(b["out"], non_blocking=True)
-            b["ev_out"].record(self.s_out)
+        self.hs.decode(0, self.h_q, self.h_tables, self.h_lens, self.scale, out, h_k=self.h_k, h_v=self.h_v,
+                       h_slot_mapping=self.h_slots)
 
     def finish_e2e(self):
         """Make the current stream wait for every copy still in flight (called inside the timed region)."""
-        main = torch.cuda.current_stream(self.dev)
-        for b in self.bufs:
-            main.wait_event(b["ev_out"])
+        self.hs.flush()
 
     def h_out_check(self):
         """Result of the resident path, on the host: the end-to-end path must deliver the same bits."""
@@ -216,6 +190,9 @@ class DecodeWorkload:
         return h2d, self.h_out.numel() * self.h_out.element_size()
 
     def close(self):
+        if getattr(self, "hs", None) is not None:
+            self.hs.close()
+            self.hs = None
         self.pool.close()
 
 
@@ -647,7 +624,7 @@ def main():
         if e2e_count[0] == args.steps:
             wl.finish_e2e()                              # the last D2H copies end inside the timed region
     ms_e2e = timed_loop(e2e_step, args.steps, device, dist)
-    assert torch.equal(wl.bufs[0]["h_out"], wl.h_out_check()) and torch.equal(wl.bufs[1]["h_out"], wl.bufs[0]["h_out"])
+    assert torch.equal(wl.h_outs[0], wl.h_out_check()) and torch.equal(wl.h_outs[1], wl.h_outs[0])
 
     step_bytes = wl.decode_bytes + wl.write_bytes
     value = whole_job_gbs(step_bytes, args.steps, ms, world)

@@ -236,6 +236,41 @@ EKV_API ekv_status_t ekv_attn_decode_two_tensor(ekv_pool_t *pool, int32_t layer,
                                                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * ekv_hoststep_* -- one decode step of a layer driven from HOST buffers (the scheduler of the paper's
+ * engine lives on the host: "Controller" acts "at scheduler step boundaries", and every step hands the
+ * attention kernel new rows, slot mappings, block tables and lengths).  The object owns `depth` sets of
+ * device staging buffers, the decode workspace, two copy streams and their events; all of it is
+ * allocated by ekv_hoststep_create, a step allocates nothing.
+ *
+ * ekv_hoststep_decode enqueues, for one step,
+ *     host -> device copies of the inputs | ekv_write_kv (unless h_k, h_v, h_slot_mapping are all NULL)
+ *     | ekv_attn_decode | device -> host copy of the result
+ * with the kernels on `stream` and the copies on the object's own streams, so that with depth >= 2 the
+ * copy-in of step i+1 and the copy-out of step i-1 overlap the kernels of step i.  It returns without
+ * synchronising.  Results are exactly those of ekv_write_kv + ekv_attn_decode on the same data.
+ *   h_q, h_out: HOST bf16 [B, num_q_heads, head_dim].  h_k, h_v: HOST bf16 [B, num_kv_heads, head_dim].
+ *   h_slot_mapping: HOST int64 [B].  h_block_tables: HOST int32 [B, max_blocks_per_seq].
+ *   h_seq_lens: HOST int32 [B].  Use pinned (page-locked) memory: copies from pageable memory are
+ *   staged by the driver and do not overlap.  Every host buffer must stay valid and unmodified until
+ *   the step has finished; h_out holds the result once the work enqueued by ekv_hoststep_flush (or a
+ *   later step on the same set) has completed.
+ *   B <= max_batch and max_blocks_per_seq <= the value given at creation, else EKV_ERR_INVALID.
+ * ekv_hoststep_flush makes `stream` wait for every copy-out still in flight; synchronise `stream`
+ * afterwards to read the results on the host.
+ * The object refers to the pool: destroy it before the pool.  Calls on one object must not run
+ * concurrently.  ekv_hoststep_destroy synchronises the device.
+ */
+typedef struct ekv_hoststep ekv_hoststep_t;
+EKV_API ekv_status_t ekv_hoststep_create(ekv_pool_t *pool, int32_t max_batch, int32_t max_blocks_per_seq, int32_t depth,
+                                         ekv_hoststep_t **out);
+EKV_API ekv_status_t ekv_hoststep_destroy(ekv_hoststep_t *step);
+EKV_API ekv_status_t ekv_hoststep_decode(ekv_hoststep_t *step, int32_t layer, const void *h_q, const void *h_k, const void *h_v,
+                                         const int64_t *h_slot_mapping, const int32_t *h_block_tables,
+                                         int32_t max_blocks_per_seq, const int32_t *h_seq_lens, int32_t B, float scale,
+                                         void *h_out, void *stream);
+EKV_API ekv_status_t ekv_hoststep_flush(ekv_hoststep_t *step, void *stream);
+
+/*
  * ekv_attn_prefill_chunk -- causal attention of a prompt chunk over its cached prefix plus itself
  * (chunked prefill: "The Decisive Test", "Why the penalty is small": chunking splits the same
  * work across steps).  Request r owns query rows cu_q_lens[r] .. cu_q_lens[r+1]-1 (c_r rows) and

@@ -14,4 +14,6 @@ from ._binding import (  # noqa: F401,E402
     ekv_blockpool_alloc, ekv_blockpool_create, ekv_blockpool_destroy, ekv_blockpool_drain_commit, ekv_blockpool_drain_plan,
     ekv_blockpool_free, ekv_blockpool_gate_elastic, ekv_blockpool_stats, ekv_controller_create, ekv_controller_decide,
     ekv_controller_destroy, ekv_controller_stats, ekv_move_blocks)
-from .pool import Pool  # noqa: F401,E402
+from ._binding import (  # noqa: F401,E402
+    ekv_hoststep_create, ekv_hoststep_decode, ekv_hoststep_destroy, ekv_hoststep_flush)
+from .pool import HostStep, Pool  # noqa: F401,E402

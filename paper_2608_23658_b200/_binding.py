@@ -115,6 +115,10 @@ def load_library():
         "ekv_attn_decode_two_tensor": (i32, [vp, i32, vp, i64, vp, vp, vp, i32, vp, i32, f32, vp, sz, vp]),
         "ekv_attn_decode_static_scratch": (i32, [vp, i32, vp, vp, vp, i32, vp, i32, f32, vp]),
         "ekv_attn_prefill_chunk": (i32, [vp, i32, vp, vp, vp, i32, vp, vp, vp, i32, f32, vp]),
+        "ekv_hoststep_create": (i32, [vp, i32, i32, i32, ctypes.POINTER(vp)]),
+        "ekv_hoststep_destroy": (i32, [vp]),
+        "ekv_hoststep_decode": (i32, [vp, i32, vp, vp, vp, vp, vp, i32, vp, i32, f32, vp, vp]),
+        "ekv_hoststep_flush": (i32, [vp, vp]),
         "ekv_poll_status": (i32, [vp]),
         "ekv_blockpool_create": (i32, [i64, i64, ctypes.POINTER(vp)]),
         "ekv_blockpool_destroy": (i32, [vp]),
@@ -260,6 +264,32 @@ def ekv_attn_decode_static_scratch(pool: int, layer: int, q, out, block_tables, 
     _check(load_library().ekv_attn_decode_static_scratch(pool, layer, _dptr(q), _dptr(out), _dptr(block_tables),
                                                          max_blocks, _dptr(seq_lens), B, float(scale),
                                                          _stream(stream)))
+
+
+def ekv_hoststep_create(pool: int, max_batch: int, max_blocks_per_seq: int, depth: int = 2) -> int:
+    out = ctypes.c_void_p()
+    _check(load_library().ekv_hoststep_create(pool, max_batch, max_blocks_per_seq, depth, ctypes.byref(out)))
+    return out.value
+
+
+def ekv_hoststep_destroy(step: int):
+    _check(load_library().ekv_hoststep_destroy(step))
+
+
+def ekv_hoststep_decode(step: int, layer: int, h_q, h_k, h_v, h_slot_mapping, h_block_tables, h_seq_lens, scale: float, h_out,
+                        stream=None):
+    """One decode step from HOST tensors (pinned for overlap); h_k / h_v / h_slot_mapping may all be None."""
+    B = int(h_seq_lens.shape[0])
+    max_blocks = int(h_block_tables.shape[1])
+    for t in (h_q, h_k, h_v, h_slot_mapping, h_block_tables, h_seq_lens, h_out):
+        assert t is None or not t.is_cuda, "ekv_hoststep_decode takes host tensors"
+    _check(load_library().ekv_hoststep_decode(step, layer, _dptr(h_q), _dptr(h_k), _dptr(h_v), _dptr(h_slot_mapping),
+                                              _dptr(h_block_tables), max_blocks, _dptr(h_seq_lens), B, float(scale),
+                                              _dptr(h_out), _stream(stream)))
+
+
+def ekv_hoststep_flush(step: int, stream=None):
+    _check(load_library().ekv_hoststep_flush(step, _stream(stream)))
 
 
 def ekv_attn_prefill_chunk(pool: int, layer: int, q, out, block_tables, cu_q_lens, cu_q_lens_host, seq_lens,

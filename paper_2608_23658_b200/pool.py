@@ -107,3 +107,31 @@ class Pool:
         B.ekv_attn_prefill_chunk(self.handle, layer, q, out, block_tables, cu_q_lens, cu_q_lens_host, seq_lens,
                                  scale, stream)
         return out
+
+
+class HostStep:
+    """Decode steps driven from pinned host tensors (ekv_hoststep_*): copies in, write_kv + decode, copy out,
+    double-buffered on the library's own copy streams.  Close it before its pool."""
+
+    def __init__(self, pool: Pool, max_batch: int, max_blocks_per_seq: int, depth: int = 2):
+        self.pool = pool
+        self.handle = B.ekv_hoststep_create(pool.handle, max_batch, max_blocks_per_seq, depth)
+
+    def decode(self, layer, h_q, h_block_tables, h_seq_lens, scale, h_out, h_k=None, h_v=None, h_slot_mapping=None,
+               stream=None):
+        B.ekv_hoststep_decode(self.handle, layer, h_q, h_k, h_v, h_slot_mapping, h_block_tables, h_seq_lens, scale, h_out,
+                              stream)
+
+    def flush(self, stream=None):
+        B.ekv_hoststep_flush(self.handle, stream)
+
+    def close(self):
+        if self.handle:
+            B.ekv_hoststep_destroy(self.handle)
+            self.handle = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
