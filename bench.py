@@ -445,8 +445,22 @@ def measure_write_kv(device, peaks):
                 ts.append(e0.elapsed_time(e1))
             ms = statistics.median(ts)
             gbs = I.write_algorithmic_bytes(T, s) / ms / 1e6
+            # the same number of bytes moved by one plain device copy, timed the same way: what a launch of this
+            # size can reach at all (the measured peak is for a 2 GiB copy)
+            src = torch.cat([k.view(-1), v.view(-1)])
+            dst = torch.empty_like(src)
+            tc = []
+            for _ in range(7):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                dst.copy_(src)
+                e1.record()
+                torch.cuda.synchronize(device)
+                tc.append(e0.elapsed_time(e1))
             res[f"tokens_{T}"] = {"ms": round(ms, 4), "gbs_read_plus_write": round(gbs, 1),
-                                  "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}
+                                  "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
+                                  "plain_copy_same_bytes_ms": round(statistics.median(tc), 4)}
         finally:
             pool.close()
     res["workload"] = "slot-mapped write of K and V rows, 8 kv heads x 128 channels, blocks scattered over the pool"
@@ -555,6 +569,8 @@ def main():
     ap.add_argument("--prefill-only", type=int, default=0, metavar="PROMPT_LEN",
                     help="profiling aid: run only the prefill-chunk measurement on a prompt of this length "
                          "(one-shot and in 4 chunks) and print its JSON")
+    ap.add_argument("--write-kv-only", action="store_true",
+                    help="profiling aid: run only the ekv_write_kv measurement (8192 and 32768 tokens) and print its JSON")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -579,6 +595,9 @@ def main():
     if args.prefill_only:
         n = args.prefill_only
         print(json.dumps({"prefill": measure_prefill(device, peaks, reps=2, prompt_len=n, chunks=(n // 4, n))}), flush=True)
+        return
+    if args.write_kv_only:
+        print(json.dumps({"write_kv": measure_write_kv(device, peaks)}), flush=True)
         return
     cfg = I.C2
     wl = DecodeWorkload(cfg, device, args.batch)

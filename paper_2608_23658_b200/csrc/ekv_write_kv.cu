@@ -14,7 +14,7 @@ static constexpr int kWriteUnroll = 4;
 __global__ void __launch_bounds__(kWriteThreads) write_kv_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ k,
                                                                  const uint4 *__restrict__ v,
                                                                  const long long *__restrict__ slot_mapping, int T,
-                                                                 int num_kv_heads, int block_size, int pieces_per_row,
+                                                                 int num_kv_heads, int block_size, int block_shift, int pieces_per_row,
                                                                  long long block_stride_pieces,
                                                                  const long long *__restrict__ live_ptr, unsigned *status) {
     const long long live = *live_ptr;
@@ -26,25 +26,29 @@ __global__ void __launch_bounds__(kWriteThreads) write_kv_kernel(uint4 *__restri
     for (long long base = (long long)blockIdx.x * chunk + threadIdx.x; base < total + threadIdx.x; base += (long long)gridDim.x * chunk) {
         uint4 val[kWriteUnroll];
         long long dst[kWriteUnroll];
+        // one 64-bit division per trip; the pieces of the trip are then located with 32-bit arithmetic
+        const long long i0 = base / token_pieces;
+        const int rem0 = (int)(base - i0 * token_pieces);
 #pragma unroll
         for (int u = 0; u < kWriteUnroll; ++u) {
-            const long long idx = base + (long long)u * kWriteThreads;
             dst[u] = -1;
-            if (idx >= total) continue;
-            const int i = (int)(idx / token_pieces);
-            const int rem = (int)(idx - (long long)i * token_pieces);
+            if (base + (long long)u * kWriteThreads >= total) continue;
+            const int r = rem0 + u * kWriteThreads;
+            const int di = r / token_pieces;
+            const int rem = r - di * token_pieces;
+            const long long i = i0 + di;
             const int kv = rem >= row_pieces;
             const int hp = rem - kv * row_pieces;  // head * pieces_per_row + piece
             const int h = hp / pieces_per_row, c = hp - h * pieces_per_row;
             const long long s = slot_mapping[i];
             if (s < 0) continue;
-            const long long n = s / block_size;
-            const int t = (int)(s - n * block_size);
+            const long long n = s >> block_shift;  // block_size is a power of two (checked at pool creation)
+            const int t = (int)(s & (block_size - 1));
             if (n >= live) {
                 if (rem == 0) atomicOr(status, EKV_DEV_FLAG_OOB);
                 continue;
             }
-            val[u] = (kv ? v : k)[(long long)i * row_pieces + hp];
+            val[u] = (kv ? v : k)[i * row_pieces + hp];
             dst[u] = n * block_stride_pieces + (((long long)(kv * num_kv_heads + h) * block_size + t) * pieces_per_row) + c;
         }
 #pragma unroll
@@ -67,13 +71,15 @@ extern "C" ekv_status_t ekv_write_kv(ekv_pool_t *pool, int32_t layer, const void
     }
     if (T == 0) return EKV_OK;
     const int pieces_per_row = pool->desc.head_dim * 2 / 16;
+    int block_shift = 0;
+    while ((1 << block_shift) < pool->desc.block_size) ++block_shift;
     const long long total = (long long)T * 2 * pool->desc.num_kv_heads * pieces_per_row;
     long long blocks = (total + kWriteThreads * kWriteUnroll - 1) / (kWriteThreads * kWriteUnroll);
-    const long long cap = (long long)pool->sm_count * 8;  // 8 CTAs of 256 threads per SM: one full wave
+    const long long cap = (long long)pool->sm_count * 64;
     if (blocks > cap) blocks = cap;
     write_kv_kernel<<<(unsigned)blocks, kWriteThreads, 0, (cudaStream_t)stream>>>(
         (uint4 *)pool->layer_base(layer), (const uint4 *)k, (const uint4 *)v, (const long long *)slot_mapping, T,
-        pool->desc.num_kv_heads, pool->desc.block_size, pieces_per_row, (long long)(pool->block_stride / 16), pool->d_live,
+        pool->desc.num_kv_heads, pool->desc.block_size, block_shift, pieces_per_row, (long long)(pool->block_stride / 16), pool->d_live,
         pool->d_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_write_kv launch");
