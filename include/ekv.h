@@ -368,6 +368,17 @@ EKV_API ekv_status_t ekv_controller_destroy(ekv_controller_t *ctrl);
 EKV_API ekv_action_t ekv_controller_decide(ekv_controller_t *ctrl, int32_t next_prefill_tokens);
 EKV_API ekv_status_t ekv_controller_stats(const ekv_controller_t *ctrl, ekv_controller_stats_t *out);
 
+/*
+ * ekv_selftest_bounded_wait -- ours (error handling; the paper has no counterpart).  Every wait inside
+ * the kernels is bounded: when it runs out, the kernel latches EKV_ERR_TIMEOUT, finishes, and the
+ * context stays usable.  This call runs that path on purpose and harmlessly: it enqueues on `stream`
+ * one small kernel that waits, with the kernels' own wait routine and a limit of limit_us microseconds
+ * (1 .. 100000), on a barrier that nothing arrives on.  After the stream has been synchronised
+ * ekv_poll_status returns EKV_ERR_TIMEOUT once, and every other call keeps working.
+ * waited_ns_device: DEVICE uint64, or NULL; receives how long the wait lasted.
+ */
+EKV_API ekv_status_t ekv_selftest_bounded_wait(ekv_pool_t *pool, int32_t limit_us, uint64_t *waited_ns_device, void *stream);
+
 /* Non-blocking read-and-clear of the status latched by kernels (EKV_OK, EKV_ERR_BLOCK_OOB or
  * EKV_ERR_TIMEOUT; the latter wins).  Meaningful after the launching stream was synchronised. */
 EKV_API ekv_status_t ekv_poll_status(ekv_pool_t *pool);

@@ -15,5 +15,5 @@ from ._binding import (  # noqa: F401,E402
     ekv_blockpool_free, ekv_blockpool_gate_elastic, ekv_blockpool_stats, ekv_controller_create, ekv_controller_decide,
     ekv_controller_destroy, ekv_controller_stats, ekv_move_blocks)
 from ._binding import (  # noqa: F401,E402
-    ekv_hoststep_create, ekv_hoststep_decode, ekv_hoststep_destroy, ekv_hoststep_flush)
+    ekv_hoststep_create, ekv_hoststep_decode, ekv_hoststep_destroy, ekv_hoststep_flush, ekv_selftest_bounded_wait)
 from .pool import HostStep, Pool  # noqa: F401,E402

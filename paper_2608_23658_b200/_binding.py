@@ -119,6 +119,7 @@ def load_library():
         "ekv_hoststep_destroy": (i32, [vp]),
         "ekv_hoststep_decode": (i32, [vp, i32, vp, vp, vp, vp, vp, i32, vp, i32, f32, vp, vp]),
         "ekv_hoststep_flush": (i32, [vp, vp]),
+        "ekv_selftest_bounded_wait": (i32, [vp, i32, vp, vp]),
         "ekv_poll_status": (i32, [vp]),
         "ekv_blockpool_create": (i32, [i64, i64, ctypes.POINTER(vp)]),
         "ekv_blockpool_destroy": (i32, [vp]),
@@ -264,6 +265,11 @@ def ekv_attn_decode_static_scratch(pool: int, layer: int, q, out, block_tables, 
     _check(load_library().ekv_attn_decode_static_scratch(pool, layer, _dptr(q), _dptr(out), _dptr(block_tables),
                                                          max_blocks, _dptr(seq_lens), B, float(scale),
                                                          _stream(stream)))
+
+
+def ekv_selftest_bounded_wait(pool: int, limit_us: int, waited_ns=None, stream=None):
+    """Runs the kernels' bounded wait until it gives up (nothing arrives); latches EKV_ERR_TIMEOUT. Harmless."""
+    _check(load_library().ekv_selftest_bounded_wait(pool, int(limit_us), _dptr(waited_ns), _stream(stream)))
 
 
 def ekv_hoststep_create(pool: int, max_batch: int, max_blocks_per_seq: int, depth: int = 2) -> int:
