@@ -14,7 +14,7 @@ static constexpr int kWriteUnroll = 4;
 __global__ void __launch_bounds__(kWriteThreads) write_kv_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ k,
                                                                  const uint4 *__restrict__ v,
                                                                  const long long *__restrict__ slot_mapping, int T,
-                                                                 int num_kv_heads, int block_size, int block_shift, int pieces_per_row,
+                                                                 int num_kv_heads, int block_size, int block_shift, int pieces_per_row, int row_shift, int token_shift,
                                                                  long long block_stride_pieces,
                                                                  const long long *__restrict__ live_ptr, unsigned *status) {
     const long long live = *live_ptr;
@@ -34,12 +34,18 @@ __global__ void __launch_bounds__(kWriteThreads) write_kv_kernel(uint4 *__restri
             dst[u] = -1;
             if (base + (long long)u * kWriteThreads >= total) continue;
             const int r = rem0 + u * kWriteThreads;
-            const int di = r / token_pieces;
-            const int rem = r - di * token_pieces;
+            int di, rem;
+            if (token_shift >= 0) {  // pieces per token a power of two (kv-head count is): no division
+                di = r >> token_shift;
+                rem = r & (token_pieces - 1);
+            } else {
+                di = r / token_pieces;
+                rem = r - di * token_pieces;
+            }
             const long long i = i0 + di;
             const int kv = rem >= row_pieces;
             const int hp = rem - kv * row_pieces;  // head * pieces_per_row + piece
-            const int h = hp / pieces_per_row, c = hp - h * pieces_per_row;
+            const int h = hp >> row_shift, c = hp & (pieces_per_row - 1);  // pieces_per_row is 8 or 16
             const long long s = slot_mapping[i];
             if (s < 0) continue;
             const long long n = s >> block_shift;  // block_size is a power of two (checked at pool creation)
@@ -71,15 +77,19 @@ extern "C" ekv_status_t ekv_write_kv(ekv_pool_t *pool, int32_t layer, const void
     }
     if (T == 0) return EKV_OK;
     const int pieces_per_row = pool->desc.head_dim * 2 / 16;
-    int block_shift = 0;
+    int block_shift = 0, row_shift = 0, token_shift = -1;
     while ((1 << block_shift) < pool->desc.block_size) ++block_shift;
+    while ((1 << row_shift) < pieces_per_row) ++row_shift;
+    const int token_pieces = 2 * pool->desc.num_kv_heads * pieces_per_row;
+    if ((token_pieces & (token_pieces - 1)) == 0)
+        for (token_shift = 0; (1 << token_shift) < token_pieces;) ++token_shift;
     const long long total = (long long)T * 2 * pool->desc.num_kv_heads * pieces_per_row;
     long long blocks = (total + kWriteThreads * kWriteUnroll - 1) / (kWriteThreads * kWriteUnroll);
     const long long cap = (long long)pool->sm_count * 64;
     if (blocks > cap) blocks = cap;
     write_kv_kernel<<<(unsigned)blocks, kWriteThreads, 0, (cudaStream_t)stream>>>(
         (uint4 *)pool->layer_base(layer), (const uint4 *)k, (const uint4 *)v, (const long long *)slot_mapping, T,
-        pool->desc.num_kv_heads, pool->desc.block_size, block_shift, pieces_per_row, (long long)(pool->block_stride / 16), pool->d_live,
+        pool->desc.num_kv_heads, pool->desc.block_size, block_shift, pieces_per_row, row_shift, token_shift, (long long)(pool->block_stride / 16), pool->d_live,
         pool->d_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_write_kv launch");
