@@ -43,3 +43,19 @@ def test_status_strings_and_no_device_error():
             assert e.status == ekv.Status.ERR_CUDA
         else:
             raise AssertionError("pool creation succeeded without a CUDA device")
+
+
+def test_header_is_plain_c_and_usable_from_a_c_program(tmp_path):
+    """include/ekv.h compiles as strict C99 and a C program drives the host-side calls (block pool, controller,
+    status strings, NULL handling) through the shared library."""
+    import shutil
+    import subprocess
+    cc = shutil.which("gcc") or shutil.which("cc")
+    assert cc, "a C compiler is part of this build's toolchain"
+    exe = str(tmp_path / "c_consumer")
+    libdir = os.path.dirname(ekv.library_path())
+    subprocess.run([cc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I" + os.path.join(ROOT, "include"),
+                    os.path.join(ROOT, "tests", "c_consumer.c"), "-o", exe, "-L" + libdir, "-lekv",
+                    "-Wl,-rpath," + libdir], check=True)
+    out = subprocess.run([exe], check=True, capture_output=True, text=True).stdout
+    assert out.strip() == "ok", out
