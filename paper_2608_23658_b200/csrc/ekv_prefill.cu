@@ -37,6 +37,8 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     const int group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     const bool use_tc = !force_mma && pool->desc.head_dim == 128 && group % 2 == 0 && scale > 0.f;
     const int bm = use_tc ? tc::kBM : kPmBM;
+    PrefillParams p;
+    p.n_prefix = R <= kPrefixMax ? 1 : 0;
     long long q_tiles = 0;
     for (int r = 0; r < R; ++r) {
         const int c = cu_q_lens_host[r + 1] - cu_q_lens_host[r];
@@ -44,14 +46,16 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
             set_error("ekv_attn_prefill_chunk: cu_q_lens decreases at request %d", r);
             return EKV_ERR_INVALID;
         }
+        if (p.n_prefix) p.tile_prefix[r] = (int)q_tiles;
         q_tiles += (c + bm - 1) / bm;
+        if (q_tiles > 0x7fffffffLL) break;
     }
+    if (p.n_prefix && q_tiles <= 0x7fffffffLL) p.tile_prefix[R] = (int)q_tiles;
     if (q_tiles == 0) return EKV_OK;
     if (q_tiles > 0x7fffffffLL) {
         set_error("ekv_attn_prefill_chunk: too many query tiles");
         return EKV_ERR_INVALID;
     }
-    PrefillParams p;
     p.q = (const __nv_bfloat16 *)q;
     p.out = (__nv_bfloat16 *)out;
     p.block_tables = block_tables;

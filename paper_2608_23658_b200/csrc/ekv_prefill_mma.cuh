@@ -27,7 +27,43 @@ struct PrefillParams {
     int max_blocks, num_q_heads, num_kv_heads, group, R;
     float scale_log2;
     unsigned long long *trace;  // debug builds only (EKV_TC_TRACE): per-role timestamps of one CTA
+    // tile_prefix[r] = query tiles of requests 0..r-1 (filled by the host when R <= kPrefixMax, else n_prefix = 0):
+    // lets a CTA find its request by bisection in the parameter bank instead of walking cu_q_lens
+    int n_prefix;
+    int tile_prefix[257];
 };
+static constexpr int kPrefixMax = 256;
+
+// Which request owns query tile `tile_idx` (tiles of `bm` rows, requests in order)?  Returns false if none.
+__device__ __forceinline__ bool find_request(const PrefillParams &p, int tile_idx, int bm, int &req, int &first_tile, int &q0,
+                                             int &c_r) {
+    if (p.n_prefix) {
+        if (tile_idx >= p.tile_prefix[p.R]) return false;
+        int lo = 0, hi = p.R;  // invariant: tile_prefix[lo] <= tile_idx < tile_prefix[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (p.tile_prefix[mid] <= tile_idx) lo = mid;
+            else hi = mid;
+        }
+        req = lo;
+        first_tile = p.tile_prefix[lo];
+        q0 = p.cu_q_lens[req];
+        c_r = p.cu_q_lens[req + 1] - q0;
+        return true;
+    }
+    int acc = 0;
+    for (req = 0; req < p.R; ++req) {
+        q0 = p.cu_q_lens[req];
+        c_r = p.cu_q_lens[req + 1] - q0;
+        const int nt = (c_r + bm - 1) / bm;
+        if (tile_idx < acc + nt) {
+            first_tile = acc;
+            return true;
+        }
+        acc += nt;
+    }
+    return false;
+}
 
 static constexpr int kPmBM = 64;      // query rows per CTA
 static constexpr int kPmBN = 64;      // keys per tile
@@ -50,14 +86,7 @@ __global__ void __launch_bounds__(128, 2) prefill_mma_kernel(const __grid_consta
     const int h = blockIdx.y;
     const int g = h / p.group;
     int req = 0, acc = 0, c_r = 0, q0 = 0;
-    for (; req < p.R; ++req) {
-        q0 = p.cu_q_lens[req];
-        c_r = p.cu_q_lens[req + 1] - q0;
-        const int nt = (c_r + kPmBM - 1) / kPmBM;
-        if (tile_idx < acc + nt) break;
-        acc += nt;
-    }
-    if (req >= p.R) return;
+    if (!find_request(p, tile_idx, kPmBM, req, acc, q0, c_r)) return;
     const int row0 = (tile_idx - acc) * kPmBM;
     const int L = min(p.seq_lens[req], p.max_blocks * 16);
     const int prefix = L - c_r;

@@ -189,14 +189,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     const int head0 = 2 * pair;
     const int g = head0 / p.group;
     int req = 0, acc_tiles = 0, c_r = 0, q0 = 0;
-    for (; req < p.R; ++req) {
-        q0 = p.cu_q_lens[req];
-        c_r = p.cu_q_lens[req + 1] - q0;
-        const int nt = (c_r + kBM - 1) / kBM;
-        if (tile_idx < acc_tiles + nt) break;
-        acc_tiles += nt;
-    }
-    if (req >= p.R) return;
+    if (!find_request(p, tile_idx, kBM, req, acc_tiles, q0, c_r)) return;
     const int row0 = (tile_idx - acc_tiles) * kBM;
     const int L = min(p.seq_lens[req], p.max_blocks * 16);
     const int prefix = L - c_r;

@@ -356,6 +356,29 @@ def test_prefill_batched_ragged_requests_match_oracle(shape):
         case.close()
 
 
+@pytest.mark.parametrize("shape,R", [(I.LLAMA8B, 60), (I.TINY, 60), (I.LLAMA8B, 300)])
+def test_prefill_many_requests_find_their_tiles(shape, R):
+    """Many short requests in one call, some of them empty: every query tile must find its request (up to 256
+    requests by bisection over a prefix table in the kernel parameters, more by walking cu_q_lens)."""
+    rows = I.uniform_ints(71, 1, R, 0, 150)                  # chunk lengths, zeros included
+    rows[R // 2] = 0
+    prefix = I.uniform_ints(71, 2, R, 0, 90)
+    lengths = rows + prefix
+    need = int(I.blocks_for(lengths, 16).sum())
+    case = Case(shape, lengths.tolist(), need + 7, 72)
+    try:
+        cu = torch.cat([torch.zeros(1, dtype=torch.int64), torch.cumsum(rows, 0)]).to(torch.int32)
+        q = rand_q(73, int(cu[-1]), shape)
+        scale = 1 / math.sqrt(shape.head_dim)
+        out = case.pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, case.d_lengths, scale)
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q,
+                                         case.tables, cu, case.lengths, scale)
+        check_close(out, want, f"{R} requests, {shape}")
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
+
+
 def test_prefill_chunked_equals_one_shot_and_decode_equals_last_row():
     shape = I.LLAMA8B
     L = 1500
