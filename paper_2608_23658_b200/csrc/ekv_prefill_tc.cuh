@@ -370,15 +370,24 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         const uint32_t t_s = tmem + lane_base + col_s(x);
         const uint32_t t_o = tmem + lane_base + col_o(x);
 
-        // ---- stage this head's Q tile: my row, 16 pieces of 16 bytes, 128-byte swizzle
+        // ---- stage this head's Q tile (128-byte swizzle).  Each warp brings in the 32 rows it will own, two rows per
+        // instruction: 16 lanes cover the 256 contiguous bytes of a row, so global loads are fully coalesced
+        // (one row per lane would touch 32 cache lines per instruction and cost microseconds per CTA).
+        const int wrow0 = (warp & 3) << 5;
         {
             uint8_t *qdst = sh.ptr + kOffQ + x * kTileBytes;
-            const bool have = row < rows_here;
-            const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((size_t)(q0 + row0 + row)) * row_stride + (size_t)head * kD);
+            const int c16 = lane & 15;
+            const __nv_bfloat16 *src = p.q + ((size_t)(q0 + row0)) * row_stride + (size_t)head * kD + c16 * 8;
+            uint4 v[16];
 #pragma unroll
-            for (int c16 = 0; c16 < 16; ++c16) {
-                const uint4 v = have ? src[c16] : make_uint4(0u, 0u, 0u, 0u);
-                *reinterpret_cast<uint4 *>(qdst + (c16 >> 3) * kHalfBytes + row * 128 + (((c16 & 7) ^ (row & 7)) << 4)) = v;
+            for (int it = 0; it < 16; ++it) {
+                const int rr = wrow0 + 2 * it + (lane >> 4);
+                v[it] = rr < rows_here ? *reinterpret_cast<const uint4 *>(src + (size_t)rr * row_stride) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int it = 0; it < 16; ++it) {
+                const int rr = wrow0 + 2 * it + (lane >> 4);
+                *reinterpret_cast<uint4 *>(qdst + (c16 >> 3) * kHalfBytes + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4)) = v[it];
             }
             fence_proxy_async_smem();
             mbar_arrive(sh.bar(Q_READY));
@@ -491,27 +500,38 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             EKV_TRACE(3, j);
         }
 
-        // ---- epilogue: O / l -> bf16 -> global (row-contiguous 256 bytes per thread)
+        // ---- epilogue: O / l -> bf16 -> this head's (now idle) Q tile in shared memory -> global.  A thread holds a
+        // whole row; writing it out directly would again touch 32 cache lines per instruction.  Each warp stages its
+        // 32 rows (16-byte pieces XOR-swizzled by row: no bank conflicts either way) and writes them back two rows
+        // per instruction, 256 contiguous bytes each.  Only the warp that wrote a row reads it: __syncwarp suffices.
         if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)(n_tiles & 1), p.status, p.abort_word);
         if (ok) {
-            fence_after();
+            fence_after();  // every MMA that read this Q tile has completed (the commit covers all earlier ones)
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            __nv_bfloat16 *dst = p.out + ((size_t)(q0 + row0 + row)) * row_stride + (size_t)head * kD;
+            uint8_t *stage = sh.ptr + kOffQ + x * kTileBytes;
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
                 float ov[32];
                 tmem_ld32(ov, t_o + 32 * cc);
-                if (row < rows_here) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 v;
-                        v.x = pack_bf16x2(ov[i] * inv, ov[i + 1] * inv);
-                        v.y = pack_bf16x2(ov[i + 2] * inv, ov[i + 3] * inv);
-                        v.z = pack_bf16x2(ov[i + 4] * inv, ov[i + 5] * inv);
-                        v.w = pack_bf16x2(ov[i + 6] * inv, ov[i + 7] * inv);
-                        *reinterpret_cast<uint4 *>(dst + 32 * cc + i) = v;
-                    }
+                for (int i = 0; i < 32; i += 8) {
+                    uint4 v;
+                    v.x = pack_bf16x2(ov[i] * inv, ov[i + 1] * inv);
+                    v.y = pack_bf16x2(ov[i + 2] * inv, ov[i + 3] * inv);
+                    v.z = pack_bf16x2(ov[i + 4] * inv, ov[i + 5] * inv);
+                    v.w = pack_bf16x2(ov[i + 6] * inv, ov[i + 7] * inv);
+                    const int piece = cc * 4 + (i >> 3);
+                    *reinterpret_cast<uint4 *>(stage + row * 256 + ((piece ^ (row & 15)) << 4)) = v;
                 }
+            }
+            __syncwarp();
+            const int piece = lane & 15;
+            __nv_bfloat16 *dst = p.out + ((size_t)(q0 + row0)) * row_stride + (size_t)head * kD + piece * 8;
+#pragma unroll
+            for (int it = 0; it < 16; ++it) {
+                const int rr = wrow0 + 2 * it + (lane >> 4);
+                const uint4 v = *reinterpret_cast<const uint4 *>(stage + rr * 256 + ((piece ^ (rr & 15)) << 4));
+                if (rr < rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)rr * row_stride) = v;
             }
         }
     }
