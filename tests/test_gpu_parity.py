@@ -379,6 +379,29 @@ def test_prefill_many_requests_find_their_tiles(shape, R):
         case.close()
 
 
+@pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY])
+@pytest.mark.parametrize("mult", [4, 16])
+def test_sharp_softmax_large_scores(shape, mult):
+    """Queries 4x and 16x larger than the configs draw them: scores spread over tens of units, a row's running
+    maximum jumps far between key tiles (the rescale paths of both kernels run), and nearly all the weight sits on a
+    few keys.  Still inside the tolerance."""
+    lengths = [1500, 333, 64]
+    case = Case(shape, lengths, 140, 77)
+    try:
+        scale = 1 / math.sqrt(shape.head_dim)
+        q = (rand_q(78, 3, shape).float() * mult).to(torch.bfloat16)      # exact: a power of two
+        check_close(case.decode(q, scale), case.oracle_decode(q, scale), f"decode, q x{mult}")
+        cu = torch.tensor(np.cumsum([0] + lengths), dtype=torch.int32)
+        qp = (rand_q(79, int(cu[-1]), shape).float() * mult).to(torch.bfloat16)
+        out = case.pool.attn_prefill_chunk(0, qp.to(DEV), case.d_tables, cu.to(DEV), cu, case.d_lengths, scale)
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, qp,
+                                         case.tables, cu, case.lengths, scale)
+        check_close(out, want, f"prefill, q x{mult}")
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
+
+
 def test_prefill_chunked_equals_one_shot_and_decode_equals_last_row():
     shape = I.LLAMA8B
     L = 1500
