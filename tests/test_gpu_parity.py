@@ -402,6 +402,35 @@ def test_sharp_softmax_large_scores(shape, mult):
         case.close()
 
 
+@pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY])
+def test_scores_that_rise_along_the_sequence_force_a_rescale_at_every_tile(shape):
+    """Keys grow along the sequence so that each 16-token block scores about 2 units (log2) above the one before: a
+    row's running maximum rises by far more than the lazy-rescale threshold at every key tile, the accumulated output
+    is scaled down by 2^-16 or less each time, and nearly all the weight sits on the last visible block."""
+    L, d = 1024, shape.head_dim
+    case = Case(shape, [L], 80, 81)
+    try:
+        ramp = (torch.arange(L) // 16).float() / 64.0                      # multiples of 1/64: exact in bf16
+        K = (ramp[:, None, None] * torch.ones(1, shape.num_kv_heads, d)).to(torch.bfloat16)
+        V = case.seqs[0][1]
+        slots = I.position_slots(case.tables[0], 0, L, shape.block_size)
+        case.pool.write_kv(0, K.to(DEV), V.to(DEV), slots.to(DEV))
+        place_sequence(case.host, shape, case.tables[0], K, V)
+        scale = 1 / math.sqrt(d)
+        qmag = 8.0 * 128 / d                                               # same score slope for both head sizes
+        q = torch.full((L, shape.num_q_heads, d), qmag, dtype=torch.bfloat16)
+        cu = torch.tensor([0, L], dtype=torch.int32)
+        out = case.pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, case.d_lengths, scale)
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, d, q, case.tables, cu,
+                                         case.lengths, scale)
+        check_close(out, want, "prefill over rising scores")
+        dec = case.pool.attn_decode(0, q[-1:].to(DEV), case.d_tables, case.d_lengths, scale)
+        check_close(dec, want[-1:], "decode over rising scores")
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
+
+
 def test_prefill_chunked_equals_one_shot_and_decode_equals_last_row():
     shape = I.LLAMA8B
     L = 1500
