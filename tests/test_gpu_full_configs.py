@@ -134,6 +134,33 @@ def test_c3_mixed_chunked_prefill_step():
         pool.close()
 
 
+def test_prefill_chunk_over_a_128k_token_prefix():
+    """The last 1024-token chunk of a 131072-token prompt (8192 blocks in the table, 1024 key tiles per query tile):
+    the prefill kernel at the longest context of the configs, sampled rows against the oracle."""
+    s = I.LLAMA8B
+    Lp, c = 131072, 1024
+    pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=Lp // 16 + 96)
+    try:
+        lengths = torch.tensor([Lp])
+        tables, _ = I.assign_blocks(I.C4.seed, 21, lengths, 16, pool.info.live_blocks)
+        I.fill_pool_layer_(pool.layer_tensor(0), I.C4.seed)
+        Q = I.normal_bf16(I.C4.seed, 6, 0, c * s.num_q_heads * s.head_dim, device=DEV).view(c, s.num_q_heads, s.head_dim)
+        cu = torch.tensor([0, c], dtype=torch.int32)
+        scale = 1 / math.sqrt(s.head_dim)
+        out = pool.attn_prefill_chunk(0, Q, tables.to(DEV), cu.to(DEV), cu, lengths.to(torch.int32).to(DEV), scale)
+        again = pool.attn_prefill_chunk(0, Q, tables.to(DEV), cu.to(DEV), cu, lengths.to(torch.int32).to(DEV), scale)
+        torch.cuda.synchronize()
+        assert pool.poll_status() == ekv.Status.OK
+        assert torch.equal(out, again)
+        rows = [0, 1, 127, 128, 500, c - 1]
+        cache, ctab, clen = host_mirror(I.C4.seed, 0, tables, lengths, [0], s)
+        want = oracle.attn_prefill_chunk(cache, s.num_q_heads, s.num_kv_heads, 16, s.head_dim, Q.cpu(), ctab,
+                                         np.array([0, c]), clen, scale, rows=np.array(rows))
+        check_close(out[rows], want, "prefill over a 130048-token prefix")
+    finally:
+        pool.close()
+
+
 # ------------------------------------------------------------------ configs[3]
 
 
