@@ -53,7 +53,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_
     }
 }
 
-// ---- TMA: tiled loads global -> shared, completion on an mbarrier (no multicast) --------------
+// ---- TMA: tiled loads global -> shared, completion on an mbarrier of the issuing CTA --------------
 // 3-D tiled loads: coordinates (channel, row inside the block, block id)
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, int x, int y, int z, uint32_t bar) {
     asm volatile(
