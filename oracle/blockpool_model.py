@@ -38,8 +38,11 @@ class BlockPoolModel:
         return out
 
     def free(self, ids):
+        """True / False (nothing freed) / "state" (an id of the outstanding drain plan: nothing freed)."""
         if len(set(ids)) != len(ids) or any(i not in self.used for i in ids):
             return False
+        if self.plan and any(i in self.plan[0] or i in self.plan[1] for i in ids):
+            return "state"
         for i in ids:
             self.used.discard(i)
             (self.free_base if i < self.base else self.free_elastic).append(i)

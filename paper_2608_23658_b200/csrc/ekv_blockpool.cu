@@ -1,11 +1,12 @@
 // Host-side block pool with a gated elastic id range, the one-step-ahead controller, and the device
 // kernel that moves blocks out of the elastic range before a decommit ("drain").
 //
-// Paper, section "An Elastic KV Mechanism": the block pool is a pure integer free list; the top
-// elastic block-id range is gated so those blocks are only handed out while the elastic slice is
-// committed ("Two handles, one virtual range"); the controller commits during decode-only phases
-// and decommits at the boundary before a prefill, with hysteresis; decommitting first drains the
-// elastic blocks, syncs, then unmaps ("Controller").
+// Follows the paper's section "An Elastic KV Mechanism".  The pool is a free list of integer ids
+// and nothing else.  Ids above base_blocks belong to the elastic slice and leave the list only while
+// that slice is committed (paragraph "Two handles, one virtual range").  The controller lends the
+// slice out while steps only decode and reclaims it just before a step that prefills, waiting a few
+// quiet steps before lending again; reclaiming means: move live data off the elastic ids, wait for
+// the device, unmap (paragraph "Controller").
 #include <string.h>
 
 #include <new>
@@ -18,7 +19,7 @@ struct ekv_blockpool {
     bool admitted;                     // elastic ids may be handed out
     std::vector<int32_t> free_base;    // stack: back() is handed out next
     std::vector<int32_t> free_elastic;
-    std::vector<uint8_t> in_use;       // per id
+    std::vector<uint8_t> in_use;       // per id: 0 free, 1 allocated, 3 allocated and part of the outstanding drain plan
     int64_t elastic_in_use;
     // drain in progress: pairs handed out by ekv_blockpool_drain_plan, settled by ekv_blockpool_drain_commit
     std::vector<int32_t> drain_from, drain_to;
@@ -99,6 +100,10 @@ ekv_status_t ekv_blockpool_free(ekv_blockpool_t *bp, const int32_t *ids, int64_t
         const int64_t id = ids[i];
         if (id < 0 || id >= bp->base + bp->elastic || bp->in_use[(size_t)id] != 1) {
             for (int64_t k = 0; k < i; ++k) bp->in_use[(size_t)ids[k]] = 1;  // undo the duplicate marks
+            if (id >= 0 && id < bp->base + bp->elastic && bp->in_use[(size_t)id] == 3) {
+                set_error("ekv_blockpool_free: id %lld belongs to the outstanding drain plan; commit the drain first", (long long)id);
+                return EKV_ERR_STATE;
+            }
             set_error("ekv_blockpool_free: id %lld is not an allocated block (or is listed twice)", (long long)id);
             return EKV_ERR_INVALID;
         }
@@ -162,10 +167,11 @@ ekv_status_t ekv_blockpool_drain_plan(ekv_blockpool_t *bp, int32_t *from_ids, in
     }
     int64_t k = 0;
     for (int64_t id = bp->base; id < bp->base + bp->elastic && k < n; ++id) {
-        if (bp->in_use[(size_t)id] != 1) continue;
+        if (bp->in_use[(size_t)id] == 0) continue;
         const int32_t to = bp->free_base.back();
         bp->free_base.pop_back();
-        bp->in_use[(size_t)to] = 1;
+        bp->in_use[(size_t)to] = 3;
+        bp->in_use[(size_t)id] = 3;
         from_ids[k] = (int32_t)id;
         to_ids[k] = to;
         bp->drain_from.push_back((int32_t)id);
@@ -185,6 +191,7 @@ ekv_status_t ekv_blockpool_drain_commit(ekv_blockpool_t *bp) {
         bp->free_elastic.push_back(id);
         --bp->elastic_in_use;
     }
+    for (int32_t id : bp->drain_to) bp->in_use[(size_t)id] = 1;  // an ordinary allocated block from now on
     bp->drain_from.clear();
     bp->drain_to.clear();
     return EKV_OK;

@@ -35,8 +35,8 @@ class LibPool:
             ekv.ekv_blockpool_free(self.h, ids)
             return True
         except ekv.EkvError as e:
-            assert e.status == ekv.Status.ERR_INVALID
-            return False
+            assert e.status in (ekv.Status.ERR_INVALID, ekv.Status.ERR_STATE)
+            return False if e.status == ekv.Status.ERR_INVALID else "state"
 
     def admit(self):
         try:
@@ -162,6 +162,30 @@ def test_library_matches_model_on_random_operations(seed):
             assert st.free_base + st.free_elastic + len(set(held)) == base + elastic and len(set(held)) == len(held)
     finally:
         lib.close()
+
+
+def test_ids_of_an_outstanding_drain_plan_cannot_be_freed():
+    """Between drain_plan and drain_commit both sides of every pair belong to the plan: freeing one would let the
+    commit push the id onto a free list a second time.  Hand-worked: base 4, elastic 2; six allocations use ids
+    0..5; freeing 1 and 2 leaves two base ids free; the plan pairs 4 -> 2 and 5 -> 1 (most recently freed first)."""
+    for make in (LibPool, BlockPoolModel):
+        pool = make(4, 2)
+        assert pool.admit() is True
+        assert pool.alloc(6) == [0, 1, 2, 3, 4, 5]
+        assert pool.free([1, 2]) is True
+        assert pool.gate() == 2
+        plan = pool.drain_plan()
+        assert (list(plan[0]), list(plan[1])) == ([4, 5], [2, 1])
+        for ids in ([4], [1], [0, 5], [2, 3]):
+            assert pool.free(ids) == "state"
+        assert pool.free([0]) is True                              # an id outside the plan is still the caller's
+        pool.drain_commit()
+        assert pool.free([4]) is False                             # the elastic side is free now
+        assert pool.free([2, 1]) is True                           # the base side became ordinary allocated blocks
+        assert pool.alloc(3) == [1, 2, 0]                          # stack order: most recently freed first
+        assert pool.alloc(1) is None                               # 3 is held, the elastic ids are gated
+        if make is LibPool:
+            pool.close()
 
 
 @pytest.mark.parametrize("seed", range(4))
