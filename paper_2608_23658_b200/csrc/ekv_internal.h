@@ -31,6 +31,8 @@ struct ekv_pool {
     std::vector<uint64_t> base_handle;     // per range
     std::vector<uint64_t> elastic_handle;  // per range, valid while elastic_held
     std::vector<char> elastic_held;        // per range: the elastic handle exists
+    std::vector<char> elastic_mapped;      // per range: the elastic handle is mapped at the top of the range
+    int64_t live_limit;                    // the live limit last published to the device (host-only pools: last decided)
 
     uint64_t layer_base(int layer) const { return fused ? va[0] + (uint64_t)layer * block_bytes : va[layer]; }
 

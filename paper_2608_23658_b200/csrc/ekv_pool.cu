@@ -149,10 +149,12 @@ static ekv_status_t be_status(int rc, const char *what, int layer) {
 __global__ void set_live_kernel(long long *live, long long value) { *live = value; }
 
 ekv_status_t launch_set_live(ekv_pool *pool, long long value, cudaStream_t stream) {
-    if (pool->host_only) return EKV_OK;
-    set_live_kernel<<<1, 1, 0, stream>>>(pool->d_live, value);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail(e, "publish live limit");
+    if (!pool->host_only) {
+        set_live_kernel<<<1, 1, 0, stream>>>(pool->d_live, value);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e, "publish live limit");
+    }
+    pool->live_limit = value;
     return EKV_OK;
 }
 
@@ -203,7 +205,7 @@ static double now_ms() {
 static void teardown(ekv_pool *p) {
     const uint64_t layer_bytes = p->base_bytes + p->elastic_bytes;  // bytes of one range
     for (size_t l = 0; l < p->va.size(); ++l) {
-        if (p->grown && p->elastic_held[l]) p->be.unmap(p->be.user, p->va[l] + p->base_bytes, p->elastic_bytes);
+        if (p->elastic_mapped[l]) p->be.unmap(p->be.user, p->va[l] + p->base_bytes, p->elastic_bytes);
         if (p->elastic_held[l]) p->be.release(p->be.user, p->elastic_handle[l]);
         if (p->base_handle[l] != ~0ull) {
             p->be.unmap(p->be.user, p->va[l], p->base_bytes);
@@ -216,9 +218,27 @@ static void teardown(ekv_pool *p) {
     if (p->h_status) cudaFreeHost(p->h_status);
 }
 
+// Undo of a grow that failed part of the way: unmap what it mapped, release what it created.  The error
+// text of the failure is kept.
+static void unmap_elastic_after_failure(ekv_pool *p, const std::vector<char> &mapped, const std::vector<char> &created) {
+    char keep[sizeof g_err];
+    memcpy(keep, g_err, sizeof keep);
+    for (int l = 0; l < p->num_ranges; ++l) {
+        if (mapped[l]) {
+            p->be.unmap(p->be.user, p->va[l] + p->base_bytes, p->elastic_bytes);
+            p->elastic_mapped[l] = 0;
+        }
+        if (created[l]) {
+            p->be.release(p->be.user, p->elastic_handle[l]);
+            p->elastic_held[l] = 0;
+        }
+    }
+    memcpy(g_err, keep, sizeof keep);
+}
+
 // Map (creating where not held) the elastic handle of every layer.  On failure everything this
-// call mapped or created is undone.
-static ekv_status_t map_elastic(ekv_pool *p) {
+// call mapped or created is undone.  `created_out` (may be NULL) receives which handles this call created.
+static ekv_status_t map_elastic(ekv_pool *p, std::vector<char> *created_out = nullptr) {
     const int L = p->num_ranges;
     std::vector<char> created(L, 0), mapped(L, 0);
     ekv_status_t st = EKV_OK;
@@ -235,20 +255,11 @@ static ekv_status_t map_elastic(ekv_pool *p) {
         st = be_status(p->be.map(p->be.user, va, p->elastic_bytes, p->elastic_handle[l]), "map elastic handle", l);
         if (st != EKV_OK) break;
         mapped[l] = 1;
+        p->elastic_mapped[l] = 1;
         st = be_status(p->be.set_access(p->be.user, va, p->elastic_bytes, p->desc.device), "grant elastic access", l);
     }
-    if (st != EKV_OK) {
-        char keep[sizeof g_err];
-        memcpy(keep, g_err, sizeof keep);
-        for (int l = 0; l < L; ++l) {
-            if (mapped[l]) p->be.unmap(p->be.user, p->va[l] + p->base_bytes, p->elastic_bytes);
-            if (created[l]) {
-                p->be.release(p->be.user, p->elastic_handle[l]);
-                p->elastic_held[l] = 0;
-            }
-        }
-        memcpy(g_err, keep, sizeof keep);
-    }
+    if (st != EKV_OK) unmap_elastic_after_failure(p, mapped, created);
+    else if (created_out) *created_out = created;
     return st;
 }
 
@@ -305,7 +316,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
     if (d.num_layers < 1 || d.num_kv_heads < 1 || d.num_q_heads < d.num_kv_heads || d.num_q_heads % d.num_kv_heads != 0 ||
         d.num_q_heads / d.num_kv_heads > 8 || (d.head_dim != 64 && d.head_dim != 128) || d.block_size != 16 ||
         d.dtype != EKV_BF16 || d.base_blocks < 1 || d.elastic_blocks < 0 || d.device < 0 ||
-        (d.flags & ~(uint32_t)(EKV_START_GROWN | EKV_FUSED_RANGE)) != 0) {
+        (d.flags & ~(uint32_t)(EKV_START_GROWN | EKV_FUSED_RANGE | EKV_PREFILL_WARP_MMA)) != 0) {
         set_error("ekv_pool_create: unsupported geometry (layers %d, heads %d/%d, head_dim %d, block_size %d, dtype %d, "
                   "blocks %lld+%lld, flags 0x%x)",
                   d.num_layers, d.num_q_heads, d.num_kv_heads, d.head_dim, d.block_size, d.dtype, (long long)d.base_blocks,
@@ -340,6 +351,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
     p->be = be;
     p->host_only = replaced;
     p->grown = false;
+    p->live_limit = 0;
     p->d_live = nullptr;
     p->h_status = nullptr;
     p->d_status = nullptr;
@@ -388,6 +400,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
         p->base_handle.push_back(~0ull);
         p->elastic_handle.push_back(0);
         p->elastic_held.push_back(0);
+        p->elastic_mapped.push_back(0);
         uint64_t h = 0;
         st = be_status(be.create(be.user, p->base_bytes, d.device, &h), "create base handle", l);
         if (st != EKV_OK) break;
@@ -404,6 +417,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
         if (st == EKV_OK) p->grown = true;
     }
 
+    p->live_limit = p->base_blocks + (p->grown ? p->elastic_blocks : 0);
     if (st == EKV_OK && !p->host_only) {
         cudaError_t e = cudaMalloc((void **)&p->d_live, 2 * sizeof(long long));  // [0] live limit, [1] abort word
         if (e == cudaSuccess) e = cudaMemset(p->d_live, 0, 2 * sizeof(long long));
@@ -477,7 +491,7 @@ ekv_status_t ekv_pool_info(const ekv_pool_t *pool, ekv_pool_info_t *info) {
     info->num_ranges = pool->num_ranges;
     info->base_blocks = pool->base_blocks;
     info->elastic_blocks = pool->elastic_blocks;
-    info->live_blocks = pool->base_blocks + (pool->grown ? pool->elastic_blocks : 0);
+    info->live_blocks = pool->live_limit;
     info->grown = pool->grown ? 1 : 0;
     int held = 0;
     for (char c : pool->elastic_held) held |= c;
@@ -510,15 +524,28 @@ ekv_status_t ekv_grow(ekv_pool_t *pool, void *stream, uint32_t flags, double *ms
         if (e != cudaSuccess) return cuda_fail(e, "ekv_grow");
     }
     const double t1 = now_ms();
-    ekv_status_t st = map_elastic(pool);
+    std::vector<char> created;
+    ekv_status_t st = map_elastic(pool, &created);
     const double t2 = now_ms();
     if (st != EKV_OK) return st;
-    pool->grown = true;
     st = launch_set_live(pool, pool->base_blocks + pool->elastic_blocks, (cudaStream_t)stream);
     if (st == EKV_OK && !pool->host_only) {
         cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
         if (e != cudaSuccess) st = cuda_fail(e, "ekv_grow: stream sync");
     }
+    if (st != EKV_OK) {
+        // The range is mapped but the kernels were not told: back to the shrunk state.  The limit is put back
+        // first (best effort: whatever broke the stream may refuse this too; the host copy is what ekv_pool_info reports).
+        char keep[sizeof g_err];
+        memcpy(keep, g_err, sizeof keep);
+        (void)launch_set_live(pool, pool->base_blocks, (cudaStream_t)stream);
+        if (!pool->host_only) (void)cudaDeviceSynchronize();
+        pool->live_limit = pool->base_blocks;
+        memcpy(g_err, keep, sizeof keep);
+        unmap_elastic_after_failure(pool, std::vector<char>(pool->num_ranges, 1), created);
+        return st;
+    }
+    pool->grown = true;
     if (ms_out) {
         ms_out[0] = t2 - t1;
         ms_out[1] = now_ms() - t0;
@@ -546,13 +573,18 @@ ekv_status_t ekv_shrink(ekv_pool_t *pool, void *stream, uint32_t flags, double *
         e = cudaDeviceSynchronize();
         if (e != cudaSuccess) return cuda_fail(e, "ekv_shrink: device sync");
     }
+    else pool->live_limit = pool->base_blocks;
     const double t1 = now_ms();
     ekv_status_t st = EKV_OK;
     for (int l = 0; l < pool->num_ranges; ++l) {
-        ekv_status_t s1 = be_status(pool->be.unmap(pool->be.user, pool->va[l] + pool->base_bytes, pool->elastic_bytes),
-                                    "unmap elastic range", l);
-        if (s1 != EKV_OK && st == EKV_OK) st = s1;
-        if (!(flags & EKV_KEEP_PHYSICAL)) {
+        if (pool->elastic_mapped[l]) {  // a range can be unmapped already: this call may be the retry of one that failed half way
+            st = be_status(pool->be.unmap(pool->be.user, pool->va[l] + pool->base_bytes, pool->elastic_bytes), "unmap elastic range", l);
+            if (st != EKV_OK) return st;  // this range and the later ones stay mapped; the pool stays "grown" with the limit at base
+            pool->elastic_mapped[l] = 0;
+        }
+        if (!(flags & EKV_KEEP_PHYSICAL) && pool->elastic_held[l]) {
+            // The handle is dropped from the books whatever the driver answers: it is unmapped, and a second
+            // release of a handle the driver may already have let go would be worse than a leak.
             ekv_status_t s2 = be_status(pool->be.release(pool->be.user, pool->elastic_handle[l]), "release elastic handle", l);
             if (s2 != EKV_OK && st == EKV_OK) st = s2;
             pool->elastic_held[l] = 0;

@@ -18,6 +18,7 @@ class FakeVmm:
         self.fail_create_at = None        # fail the k-th create call from now (0-based)
         self.fail_map_at = None
         self.fail_access_at = None
+        self.fail_unmap_at = None
         self._next_va = 0x7000_0000_0000
         self._next_h = 101
         self.violations = []
@@ -105,6 +106,9 @@ class FakeVmm:
     def unmap(self, user, va, size):
         if va not in self.mapped or self.mapped[va][0] != size:
             return self._bad("unmap must cover exactly one whole mapping")
+        if self._tick("fail_unmap_at"):
+            self.log.append(("unmap-refused", va, size))
+            return FAIL
         del self.mapped[va]
         self.access.discard(va)
         self.log.append(("unmap", va, size))
