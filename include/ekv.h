@@ -80,8 +80,12 @@ enum {
     EKV_START_GROWN = 1u << 0,   /* ekv_pool_create: map the elastic slice right away */
     EKV_KEEP_PHYSICAL = 1u << 1, /* ekv_shrink: unmap only, keep the elastic handle (bytes survive
                                     until the next ekv_grow maps it again) */
-    EKV_FUSED_RANGE = 1u << 2    /* ekv_pool_create: ONE virtual range and two handles for all layers
-                                    instead of one range and two handles per layer (see below) */
+    EKV_FUSED_RANGE = 1u << 2,   /* ekv_pool_create: ONE virtual range and two handles for all layers
+                                    instead of one range and two handles per layer (see above) */
+    EKV_PREFILL_WARP_MMA = 1u << 3 /* ekv_pool_create: ekv_attn_prefill_chunk on this pool always runs the
+                                    warp-level (mma.sync) kernel, never a tcgen05 one.  Same results within
+                                    the stated tolerance; exists so the two kernel families can be checked
+                                    against each other in one process. */
 };
 
 typedef struct ekv_pool_desc {
@@ -92,7 +96,7 @@ typedef struct ekv_pool_desc {
     int32_t head_dim;       /* 64 or 128 */
     int32_t block_size;     /* 16 */
     int32_t dtype;          /* EKV_BF16 */
-    uint32_t flags;         /* EKV_START_GROWN */
+    uint32_t flags;         /* EKV_START_GROWN | EKV_FUSED_RANGE | EKV_PREFILL_WARP_MMA */
     int64_t base_blocks;    /* per layer, >= 1; rounded UP to whole granules */
     int64_t elastic_blocks; /* per layer, >= 0; rounded UP to whole granules */
 } ekv_pool_desc_t;
@@ -104,8 +108,10 @@ typedef struct ekv_pool_info {
     uint64_t elastic_bytes;  /* per layer, after rounding */
     int64_t base_blocks;     /* after rounding */
     int64_t elastic_blocks;  /* after rounding */
-    int64_t live_blocks;     /* base_blocks, or base_blocks + elastic_blocks while grown */
-    int32_t grown;           /* elastic slice mapped */
+    int64_t live_blocks;     /* the limit last published to the kernels: base_blocks, or base_blocks +
+                                elastic_blocks while grown */
+    int32_t grown;           /* elastic slice mapped (in every range, or -- only after an ekv_shrink that
+                                failed half way -- still in some of them) */
     int32_t physical_held;   /* elastic handles exist (mapped, or kept by EKV_KEEP_PHYSICAL) */
     int32_t num_layers;
     int32_t num_ranges;          /* virtual ranges the pool holds: num_layers, or 1 with EKV_FUSED_RANGE */
@@ -129,7 +135,7 @@ EKV_API ekv_status_t ekv_pool_destroy(ekv_pool_t *pool);
 EKV_API ekv_status_t ekv_pool_info(const ekv_pool_t *pool, ekv_pool_info_t *info);
 
 /* Device address of the layer's range; constant for the pool's life whether the elastic slice is
- * mapped or not (the paper's "the virtual range never moves").  dptr: HOST, receives a DEVICE
+ * mapped or not (the paper's point: a layer's range stays where it is).  dptr: HOST, receives a DEVICE
  * address.  Touching bytes of the elastic sub-range while it is unmapped faults the context. */
 EKV_API ekv_status_t ekv_layer_ptr(const ekv_pool_t *pool, int32_t layer, void **dptr);
 
@@ -149,8 +155,12 @@ EKV_API ekv_status_t ekv_grow(ekv_pool_t *pool, void *stream, uint32_t flags, do
  * on `stream`, synchronises the whole device (every stream that may still read elastic blocks),
  * unmaps the elastic sub-range of every layer and, unless EKV_KEEP_PHYSICAL, releases the
  * handles (the memory returns to the driver).  Precondition the library cannot check: the caller
- * no longer uses block ids >= base_blocks ("drains those blocks").  A kernel launched afterwards
+ * no longer uses block ids >= base_blocks (the drain step of "Controller").  A kernel launched afterwards
  * with such an id skips it and latches EKV_ERR_BLOCK_OOB instead of faulting.  ms_out as above.
+ * If the driver refuses to unmap some range, the call stops there and returns EKV_ERR_CUDA: ranges
+ * already unmapped stay unmapped, the others stay mapped, the pool still counts as grown
+ * (ekv_pool_info: grown = 1) while the live limit is already base_blocks, so no kernel reaches the
+ * elastic ids; calling ekv_shrink again retries the ranges that are left.
  */
 EKV_API ekv_status_t ekv_shrink(ekv_pool_t *pool, void *stream, uint32_t flags, double *ms_out);
 
@@ -166,14 +176,22 @@ EKV_API ekv_status_t ekv_shrink(ekv_pool_t *pool, void *stream, uint32_t flags, 
 EKV_API ekv_status_t ekv_write_kv(ekv_pool_t *pool, int32_t layer, const void *k, const void *v,
                           const int64_t *slot_mapping, int32_t T, void *stream);
 
-/* Bytes of scratch ekv_attn_decode needs for any call with B <= max_batch and
- * max_blocks_per_seq*block_size <= max_seq_len (rounded up to a block).  ekv_attn_prefill_chunk
- * needs none.  Returns 0 for a NULL pool. */
+/* Bytes of scratch that cover EVERY ekv_attn_decode call with 1 <= B <= max_batch and
+ * max_blocks_per_seq*block_size <= max_seq_len (rounded up to a block) -- an upper bound over all
+ * those shapes, not the need of the largest one alone (a shorter table can be cut into more key
+ * ranges than a longer one).  ekv_attn_prefill_chunk needs none.  Returns 0 for a NULL pool. */
 EKV_API size_t ekv_attn_workspace_bytes(const ekv_pool_t *pool, int32_t max_batch, int32_t max_seq_len);
+
+/* The split plan ekv_attn_decode will use for a call of exactly this shape (ours; the paper has no
+ * counterpart): keys per range, ranges per sequence at the maximum length, and the scratch that one
+ * call needs.  Any of the three HOST out-pointers may be NULL.  Depends only on the pool's geometry,
+ * the device's SM count, B and max_blocks_per_seq. */
+EKV_API ekv_status_t ekv_attn_decode_plan(const ekv_pool_t *pool, int32_t B, int32_t max_blocks_per_seq,
+                                          int32_t *chunk_tokens, int32_t *nsplit, size_t *workspace_bytes);
 
 /*
  * ekv_attn_decode -- grouped-query attention of ONE query token per sequence over that sequence's
- * cached keys/values ("the attention kernel" of "The contiguity constraint"; decode contributes
+ * cached keys/values (the kernel "The contiguity constraint" is about; decode contributes
  * one token per sequence per step, "Why the penalty is small").
  *   out[b,h,:] = sum_j softmax_j(scale * q[b,h,:].K_j) V_j ,  j = 0 .. seq_lens[b]-1,
  * where key j of sequence b is token j%block_size of block block_tables[b][j/block_size] and query
@@ -221,7 +239,8 @@ EKV_API ekv_status_t ekv_attn_decode_static_scratch(ekv_pool_t *pool, int32_t la
 
 /*
  * ekv_attn_decode_two_tensor -- the alternative the paper weighs and rejects in "The contiguity
- * constraint": "split the KV into two tensors and rewrite the kernel to read both".  Same computation
+ * constraint": keep base and elastic blocks in two separate tensors and teach the attention kernel
+ * to choose between them.  Same computation
  * and arguments as ekv_attn_decode, except that block ids 0..base_blocks-1 address the pool's base
  * range of `layer` and ids base_blocks..base_blocks+second_blocks-1 address `second_tensor`, a
  * separately allocated DEVICE buffer of second_blocks*block_bytes with the same block layout (16-byte
@@ -237,7 +256,7 @@ EKV_API ekv_status_t ekv_attn_decode_two_tensor(ekv_pool_t *pool, int32_t layer,
 
 /*
  * ekv_hoststep_* -- one decode step of a layer driven from HOST buffers (the scheduler of the paper's
- * engine lives on the host: "Controller" acts "at scheduler step boundaries", and every step hands the
+ * engine lives on the host: "Controller" acts between scheduler steps, and every step hands the
  * attention kernel new rows, slot mappings, block tables and lengths).  The object owns `depth` sets of
  * device staging buffers, the decode workspace, two copy streams and their events; all of it is
  * allocated by ekv_hoststep_create, a step allocates nothing.
@@ -290,13 +309,13 @@ EKV_API ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, con
 
 /*
  * ---- Block pool with a gated elastic id range, drain, and the one-step-ahead controller ----------
- * Paper, section "An Elastic KV Mechanism": "we gate the top elastic block-id range in the block
- * pool so those blocks are only handed out when the elastic slice is committed" (paragraph "Two
- * handles, one virtual range"); "The block pool is a pure integer free list" (section "Background
- * and Motivation"); "The controller commits the elastic slice during decode-only phases and
- * decommits it at the boundary before a prefill, with hysteresis ...  Committing grows
- * num_gpu_blocks and admits the top elastic blocks.  Decommitting first drains those blocks, syncs,
- * and then unmaps" (paragraph "Controller").
+ * Paper, section "An Elastic KV Mechanism".  Paragraph "Two handles, one virtual range": the block
+ * ids at the top of the range are gated inside the block pool, which hands them out only while the
+ * elastic slice is committed.  Section "Background and Motivation": the block pool is nothing but a
+ * free list of integers.  Paragraph "Controller": the slice is lent to the pool while the engine
+ * only decodes and taken back at the step boundary before a prefill, with hysteresis; a commit
+ * raises the number of usable blocks and admits the top ids; a decommit moves live data out of
+ * those ids, waits for the device, and only then unmaps.
  *
  * All of this is host-side bookkeeping (no CUDA call) except ekv_move_blocks.  Intended order of a
  * decommit:  ekv_blockpool_gate_elastic -> ekv_blockpool_drain_plan -> ekv_move_blocks (+ the caller
@@ -324,7 +343,8 @@ EKV_API ekv_status_t ekv_blockpool_destroy(ekv_blockpool_t *bp);
  * elastic ids only while admitted and only once no base id is free. */
 EKV_API ekv_status_t ekv_blockpool_alloc(ekv_blockpool_t *bp, int64_t n, int32_t *ids_out);
 /* Returns ids to the free list.  Any id that is not currently allocated (or appears twice) fails the
- * whole call with EKV_ERR_INVALID and frees nothing. */
+ * whole call with EKV_ERR_INVALID and frees nothing; so does, with EKV_ERR_STATE, an id on either
+ * side of an outstanding drain plan. */
 EKV_API ekv_status_t ekv_blockpool_free(ekv_blockpool_t *bp, const int32_t *ids, int64_t n);
 /* After ekv_grow: elastic ids may be handed out; num_gpu_blocks grows. */
 EKV_API ekv_status_t ekv_blockpool_admit_elastic(ekv_blockpool_t *bp);

@@ -13,6 +13,7 @@ EKV_BF16 = 0
 EKV_START_GROWN = 1
 EKV_KEEP_PHYSICAL = 2
 EKV_FUSED_RANGE = 4
+EKV_PREFILL_WARP_MMA = 8
 
 
 class Status(enum.IntEnum):
@@ -111,6 +112,7 @@ def load_library():
         "ekv_shrink": (i32, [vp, vp, u32, dblp]),
         "ekv_write_kv": (i32, [vp, i32, vp, vp, vp, i32, vp]),
         "ekv_attn_workspace_bytes": (sz, [vp, i32, i32]),
+        "ekv_attn_decode_plan": (i32, [vp, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(sz)]),
         "ekv_attn_decode": (i32, [vp, i32, vp, vp, vp, i32, vp, i32, f32, vp, sz, vp]),
         "ekv_attn_decode_two_tensor": (i32, [vp, i32, vp, i64, vp, vp, vp, i32, vp, i32, f32, vp, sz, vp]),
         "ekv_attn_decode_static_scratch": (i32, [vp, i32, vp, vp, vp, i32, vp, i32, f32, vp]),
@@ -228,6 +230,14 @@ def ekv_write_kv(pool: int, layer: int, k, v, slot_mapping, stream=None):
 
 def ekv_attn_workspace_bytes(pool: int, max_batch: int, max_seq_len: int) -> int:
     return int(load_library().ekv_attn_workspace_bytes(pool, max_batch, max_seq_len))
+
+
+def ekv_attn_decode_plan(pool: int, B: int, max_blocks_per_seq: int):
+    """Returns (keys per range, ranges per sequence, scratch bytes) of a decode call of exactly this shape."""
+    chunk, nsplit, need = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_size_t()
+    _check(load_library().ekv_attn_decode_plan(pool, B, max_blocks_per_seq, ctypes.byref(chunk), ctypes.byref(nsplit),
+                                               ctypes.byref(need)))
+    return int(chunk.value), int(nsplit.value), int(need.value)
 
 
 def ekv_attn_decode(pool: int, layer: int, q, out, block_tables, seq_lens, scale: float, workspace, stream=None):

@@ -353,28 +353,23 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeParams p)
     p.out[(size_t)bh * D + x] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
 }
 
-static int chunk_max_tokens() {
-    static int v = [] {
-        int x = 2048;
-        if (const char *e = getenv("EKV_DECODE_CHUNK_MAX")) x = atoi(e);
-        x = (x / 64) * 64;
-        return x < 64 ? 64 : (x > kChunkMaxLimit ? kChunkMaxLimit : x);
-    }();
-    return v;
+static constexpr int kChunkMin = 256;  // 4 blocks per warp: below that the fixed cost of a CTA dominates
+
+// Key ranges per (sequence, kv-head) that would fill the machine: 2 CTAs resident per SM, about 4 waves.
+static long long wanted_splits(const ekv_pool *pool, int B) {
+    const long long units = (long long)B * pool->desc.num_kv_heads;
+    const long long target = (long long)pool->sm_count * 2 * 4;
+    const long long want = (target + units - 1) / units;
+    return want < 1 ? 1 : want;
 }
 
 DecodePlan plan_decode(const ekv_pool *pool, int B, int max_blocks_per_seq) {
     const int max_len = max_blocks_per_seq * pool->desc.block_size;
-    const long long units = (long long)B * pool->desc.num_kv_heads;
-    const long long target = (long long)pool->sm_count * 2 * 4;  // CTAs: 2 per SM resident, ~4 waves
-    long long want = (target + units - 1) / units;
-    if (want < 1) want = 1;
+    const long long want = wanted_splits(pool, B);
     long long chunk = (max_len + want - 1) / want;
     chunk = (chunk + 63) / 64 * 64;
-    const int cmax = chunk_max_tokens();
-    if (chunk > cmax) chunk = cmax;
-    // at least 4 blocks per warp (256 keys) when the length allows: below that the fixed cost of a CTA dominates
-    const long long cmin = max_len >= 256 ? 256 : (max_len + 63) / 64 * 64;
+    if (chunk > kChunkMaxLimit) chunk = kChunkMaxLimit;
+    const long long cmin = max_len >= kChunkMin ? kChunkMin : (max_len + 63) / 64 * 64;
     if (chunk < cmin) chunk = cmin;
     DecodePlan plan;
     plan.chunk_tokens = (int)chunk;
@@ -462,16 +457,44 @@ static ekv_status_t dispatch_decode(ekv_pool *pool, int layer, const DecodeParam
 
 using namespace ekv;
 
+// Upper bound of plan_decode(pool, B, m).nsplit over every table width m <= max_blocks.  A shorter table can be cut
+// into MORE ranges than the longest one (the range length is rounded up to 64 keys and floored at kChunkMin), so
+// the plan of the largest shape alone is not a bound.  Three regimes of plan_decode:
+//   range length not clamped, or raised to the floor: it is >= len/want, so nsplit <= want; and it is >= kChunkMin
+//     (or covers the whole of a shorter table), so nsplit <= ceil(len / kChunkMin);
+//   range length cut down to kChunkMaxLimit: nsplit = ceil(len / kChunkMaxLimit), largest at the largest len.
+static long long nsplit_bound(const ekv_pool *pool, int B, int max_blocks) {
+    const long long max_len = (long long)max_blocks * pool->desc.block_size;
+    const long long by_floor = (max_len + kChunkMin - 1) / kChunkMin;
+    const long long by_cap = (max_len + kChunkMaxLimit - 1) / kChunkMaxLimit;
+    long long n = wanted_splits(pool, B);
+    if (n > by_floor) n = by_floor;
+    if (n < by_cap) n = by_cap;
+    return n < 1 ? 1 : n;
+}
+
 extern "C" size_t ekv_attn_workspace_bytes(const ekv_pool_t *pool, int32_t max_batch, int32_t max_seq_len) {
     if (!pool || max_batch < 1 || max_seq_len < 1) return 0;
     const int max_blocks = (max_seq_len + pool->desc.block_size - 1) / pool->desc.block_size;
     size_t need = 0;
     for (int B = 1; B <= max_batch; ++B) {
-        const DecodePlan plan = plan_decode(pool, B, max_blocks);
-        const size_t n = decode_workspace_need(pool, B, plan.nsplit);
+        const size_t n = decode_workspace_need(pool, B, (int)nsplit_bound(pool, B, max_blocks));
         if (n > need) need = n;
     }
     return need;
+}
+
+extern "C" ekv_status_t ekv_attn_decode_plan(const ekv_pool_t *pool, int32_t B, int32_t max_blocks_per_seq, int32_t *chunk_tokens,
+                                             int32_t *nsplit, size_t *workspace_bytes) {
+    if (!pool || B < 1 || B > 65535 || max_blocks_per_seq < 1 || max_blocks_per_seq > (1 << 26)) {
+        set_error("ekv_attn_decode_plan: bad argument (B=%d, max_blocks_per_seq=%d)", B, max_blocks_per_seq);
+        return EKV_ERR_INVALID;
+    }
+    const DecodePlan plan = plan_decode(pool, B, max_blocks_per_seq);
+    if (chunk_tokens) *chunk_tokens = plan.chunk_tokens;
+    if (nsplit) *nsplit = plan.nsplit;
+    if (workspace_bytes) *workspace_bytes = decode_workspace_need(pool, B, plan.nsplit);
+    return EKV_OK;
 }
 
 extern "C" ekv_status_t ekv_attn_decode(ekv_pool_t *pool, int32_t layer, const void *q, void *out,

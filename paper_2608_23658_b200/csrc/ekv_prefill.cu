@@ -1,9 +1,5 @@
 // ekv_attn_prefill_chunk: host entry point.  Validates, sizes the launch from the host copy of
 // cu_q_lens (no device synchronisation) and dispatches the kernel for the pool's head_dim.
-#include <stdio.h>
-#include <stdlib.h>
-#include <string.h>
-
 #include "ekv_internal.h"
 #include "ekv_prefill_mma.cuh"
 #include "ekv_prefill_tc.cuh"
@@ -28,12 +24,9 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
         return EKV_ERR_INVALID;
     }
     // tcgen05 kernel: head_dim 128, query heads paired inside a kv group, positive scale.  Everything
-    // else (and EKV_PREFILL_IMPL=mma, used by the tests to cross-check the two kernels) takes the
-    // warp-level MMA kernel.
-    static const bool force_mma = [] {
-        const char *e = getenv("EKV_PREFILL_IMPL");
-        return e && strcmp(e, "mma") == 0;
-    }();
+    // else (and every call on a pool created with EKV_PREFILL_WARP_MMA, which the tests use to check
+    // the two kernels against each other) takes the warp-level MMA kernel.
+    const bool force_mma = (pool->desc.flags & EKV_PREFILL_WARP_MMA) != 0;
     const int group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     const bool use_tc = !force_mma && pool->desc.head_dim == 128 && group % 2 == 0 && scale > 0.f;
     const int bm = use_tc ? tc::kBM : kPmBM;
@@ -70,26 +63,6 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     p.R = R;
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.trace = nullptr;
-#ifdef EKV_TC_TRACE
-    static unsigned long long *trace_buf = nullptr;
-    if (!trace_buf) cudaMalloc(&trace_buf, 8 * (1 + 2 * 4096));
-    cudaMemsetAsync(trace_buf, 0, 8 * (1 + 2 * 4096), (cudaStream_t)stream);
-    p.trace = trace_buf;
-#endif
-#ifdef EKV_TC_TRACE
-    if (use_tc) {
-        ekv_status_t r = tc::launch_prefill_tc(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
-        cudaStreamSynchronize((cudaStream_t)stream);
-        static unsigned long long host[12 * 8];
-        cudaMemcpy(host, p.trace, sizeof host, cudaMemcpyDeviceToHost);
-        if (getenv("EKV_TC_TRACE_PRINT"))
-            for (int w = 0; w < 12; ++w)
-                fprintf(stderr, "trace warp %2d: %9llu %9llu %9llu %9llu %9llu %9llu %9llu %9llu\n", w, host[w * 8], host[w * 8 + 1],
-                        host[w * 8 + 2], host[w * 8 + 3], host[w * 8 + 4], host[w * 8 + 5], host[w * 8 + 6], host[w * 8 + 7]);
-        return r;
-    }
-#endif
     if (use_tc) return tc::launch_prefill_tc(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
     if (pool->desc.head_dim == 128) return launch_prefill_mma<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
     return launch_prefill_mma<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);

@@ -1,6 +1,6 @@
 // Chunked-prefill attention, warp-level tensor path (mma.sync m16n8k16).  Used for head_dim 64,
 // where the query tile of the tcgen05 kernel does not apply, and as the in-library cross-check of
-// the tcgen05 kernel in the GPU tests (EKV_PREFILL_IMPL=mma).
+// the tcgen05 kernel in the GPU tests (pools created with EKV_PREFILL_WARP_MMA).
 //
 // CTA = 4 warps = 64 query rows of one (request, q-head); KV tiles of 64 tokens (4 blocks) arrive
 // through a 2-stage ring of TMA box loads (128-byte swizzle) on mbarriers.  Per warp: S(16x64) =
@@ -26,7 +26,6 @@ struct PrefillParams {
     int *abort_word;  // device word: a CTA of this launch gave up on a wait (tcgen05 kernel)
     int max_blocks, num_q_heads, num_kv_heads, group, R;
     float scale_log2;
-    unsigned long long *trace;  // debug builds only (EKV_TC_TRACE): per-role timestamps of one CTA
     // tile_prefix[r] = query tiles of requests 0..r-1 (filled by the host when R <= kPrefixMax, else n_prefix = 0):
     // lets a CTA find its request by bisection in the parameter bank instead of walking cu_q_lens
     int n_prefix;

@@ -117,27 +117,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
     cp::tcgen05_st_32x32b(taddr, r);
 }
 
-// Debug builds (EKV_TC_TRACE): every warp of CTA (0,0) accumulates cycles per phase in registers and
-// writes the totals once at the end (slot = warp*8 + phase).
-#ifdef EKV_TC_TRACE
-#define EKV_TRACE_DECL long long tr_acc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long tr_t_ = clock64();
-#define EKV_TRACE(ev, j)                          \
-    do {                                          \
-        const long long now_ = clock64();         \
-        tr_acc_[(ev) & 7] += now_ - tr_t_;        \
-        tr_t_ = now_;                             \
-    } while (0)
-#define EKV_TRACE_FLUSH                                                                              \
-    do {                                                                                             \
-        if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0)                \
-            for (int i_ = 0; i_ < 8; ++i_) p.trace[(threadIdx.x >> 5) * 8 + i_] = (unsigned long long)tr_acc_[i_]; \
-    } while (0)
-#else
-#define EKV_TRACE_DECL
-#define EKV_TRACE(ev, j) do { } while (0)
-#define EKV_TRACE_FLUSH do { } while (0)
-#endif
-
 static constexpr int kPartSteps = 6;  // PV k-steps (16 keys each) covered by the early P_PART arrival (even, 2..6)
 
 struct Shared {
@@ -243,7 +222,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     __syncthreads();
     fence_after();
     const uint32_t tmem = *sh.tmem_slot();
-    EKV_TRACE_DECL
 
     if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
@@ -287,10 +265,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 mbar_expect_tx(sh.bar(FULL + s), kTileBytes);
             }
             __syncwarp();
-            EKV_TRACE(0, j);
             if (lane < 16)
                 tma_load_3d(tile_base + s * kTileBytes + half * kHalfBytes + blk * 2048, &kvmap, 64 * half, row, my_id, sh.bar(FULL + s));
-            EKV_TRACE(1, j);
         }
     } else if (warp == 1) {
         // =========================== MMA issuer ===========================
@@ -313,7 +289,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 mma_ts_lo_dyn(tmem + col_o(x), tmem + col_s(x) + 8 * k, v_lo + ((k * 2048) >> 4), kIdescPV, (acc || k > 0) ? 1u : 0u);
         };
         bool ok = wait_warp(sh, Q_READY, 0, p.status, p.abort_word) && wait_warp(sh, K_FULL + 0, 0, p.status, p.abort_word);
-        EKV_TRACE(7, 0);
         if (ok) {
             fence_after();
             issue_qk(0, 0);
@@ -326,26 +301,22 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 const bool more = j + 1 < n_tiles;
                 ok = wait_warp(sh, V_FULL + s, (uint32_t)((j / kStages) & 1), p.status, p.abort_word);
                 if (ok && more) ok = wait_warp(sh, K_FULL + s1, (uint32_t)(((j + 1) / kStages) & 1), p.status, p.abort_word);
-                EKV_TRACE(0, j);
                 if (ok) ok = wait_warp(sh, P_PART + 0, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
                 fence_after();
                 issue_pv(0, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
                 ok = wait_warp(sh, P_READY + 0, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
-                EKV_TRACE(1, j);
                 fence_after();
                 issue_pv(0, s, true, kPartSteps, kBN / 16);
                 if (more) issue_qk(0, s1);
                 mma_commit(sh.bar(S_READY + 0));
-                EKV_TRACE(2, j);
                 ok = wait_warp(sh, P_PART + 1, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
                 fence_after();
                 issue_pv(1, s, j > 0, 0, kPartSteps);
                 ok = wait_warp(sh, P_READY + 1, (uint32_t)(j & 1), p.status, p.abort_word);
                 if (!ok) break;
-                EKV_TRACE(3, j);
                 fence_after();
                 issue_pv(1, s, true, kPartSteps, kBN / 16);
                 mma_commit(sh.bar(V_EMPTY + s));
@@ -398,11 +369,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j % kStages;
-            EKV_TRACE(4, j);
             ok = wait_warp(sh, S_READY + x, (uint32_t)(j & 1), p.status, p.abort_word);
             if (!ok) break;
             fence_after();
-            EKV_TRACE(0, j);
             const int key0 = j * kBN;
             const int bad = *sh.bad_mask(j);
             const bool need_mask = (key0 + kBN - 1 > prefix + row0) || bad != 0;
@@ -447,7 +416,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 mx3 = fmaxf(mx3, sv[i + 3]);
             }
             const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            EKV_TRACE(1, j);
             const float m_tile = mx * p.scale_log2;  // scale > 0 on this path
             // ---- lazy rescale: raise the reference max only when it is far behind
             const bool raise = m_tile > m_run + kRescaleThreshold;  // also true for the first finite tile
@@ -497,7 +465,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             cp::tcgen05_wait_st();
             fence_before();
             mbar_arrive(sh.bar(P_READY + x));
-            EKV_TRACE(3, j);
         }
 
         // ---- epilogue: O / l -> bf16 -> this head's (now idle) Q tile in shared memory -> global.  A thread holds a
@@ -547,8 +514,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         }
     }
     __syncthreads();
-    EKV_TRACE(6, 0);
-    EKV_TRACE_FLUSH;
     if (warp == 2) cp::tcgen05_dealloc(cp::cta_group_1, tmem, 512);
 }
 

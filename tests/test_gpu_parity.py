@@ -515,9 +515,6 @@ def test_elastic_toggle_bytes_pointer_and_outputs():
 def test_prefill_edge_cases_bad_ids_empty_requests_and_both_kernels_agree():
     """Out-of-range block ids inside a prompt are skipped and latched (both prefill kernels); requests with zero
     rows are legal; the tcgen05 kernel and the warp-MMA kernel agree within tolerance on the same call."""
-    import os
-    import subprocess
-    import sys
     shape = I.LLAMA8B
     pool = make_pool(shape, 128, 32, grown=False)
     try:
@@ -557,18 +554,26 @@ def test_prefill_edge_cases_bad_ids_empty_requests_and_both_kernels_agree():
         assert pool.poll_status() == ekv.Status.OK
     finally:
         pool.close()
-    # the same call through each kernel (selected by the environment when the library is first used): one
-    # process per kernel, see tests/prefill_impl_probe.py
-    import tempfile
-    probe = os.path.join(os.path.dirname(os.path.abspath(__file__)), "prefill_impl_probe.py")
-    with tempfile.TemporaryDirectory() as d:
-        outs = {}
-        for impl in ("mma", "tc"):
-            path = os.path.join(d, impl + ".pt")
-            subprocess.run([sys.executable, probe, path], check=True, env=dict(os.environ, EKV_PREFILL_IMPL=impl))
-            outs[impl] = torch.load(path)
-        diff = (outs["mma"].float() - outs["tc"].float()).abs()
-        assert diff.max().item() <= MAX_ABS and diff.mean().item() <= MEAN_ABS
+    # the same call through each kernel family (a pool created with EKV_PREFILL_WARP_MMA always takes the warp-level
+    # kernel), each against the oracle and against the other
+    outs = {}
+    for impl in ("mma", "tc"):
+        pool = ekv.Pool(num_q_heads=shape.num_q_heads, num_kv_heads=shape.num_kv_heads, head_dim=shape.head_dim,
+                        base_blocks=64, prefill_warp_mma=(impl == "mma"))
+        try:
+            case = Case(shape, [700, 45], 64, 93, pool=pool)
+            cu = torch.tensor([0, 300, 345], dtype=torch.int32)
+            q = rand_q(94, 345, shape)
+            out = pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, case.d_lengths, 0.088)
+            want = oracle.attn_prefill_chunk(case.host, 32, 8, 16, 128, q, case.tables, cu, case.lengths, 0.088)
+            check_close(out, want, impl + " prefill kernel")
+            outs[impl] = out.float().cpu()
+            assert pool.poll_status() == ekv.Status.OK
+        finally:
+            pool.close()
+    diff = (outs["mma"] - outs["tc"]).abs()
+    assert diff.max().item() <= MAX_ABS and diff.mean().item() <= MEAN_ABS
+    assert not torch.equal(outs["mma"], outs["tc"]), "two different kernels are expected to round differently somewhere"
 
 
 def test_recommit_out_of_memory_leaves_the_pool_shrunk_and_usable():

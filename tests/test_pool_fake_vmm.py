@@ -152,7 +152,7 @@ def test_failed_create_leaves_nothing_behind(vmm):
 
 def test_argument_checks_and_host_only_refusal(vmm):
     for bad in (dict(head_dim=96), dict(block_size=32), dict(num_q_heads=12, num_kv_heads=8),
-                dict(num_q_heads=72, num_kv_heads=8), dict(base_blocks=0), dict(elastic_blocks=-1), dict(flags=8)):
+                dict(num_q_heads=72, num_kv_heads=8), dict(base_blocks=0), dict(elastic_blocks=-1), dict(flags=16)):
         with pytest.raises(ekv.EkvError) as e:
             _create(**bad)
         assert e.value.status == ekv.Status.ERR_INVALID
@@ -200,3 +200,71 @@ def test_fused_range_is_one_reservation_and_two_handles_for_all_layers(vmm):
     assert len(vmm.handles) == 1 and len(vmm.mapped) == 1 and not ekv.ekv_pool_info(pool).grown
     ekv.ekv_pool_destroy(pool)
     assert not vmm.reserved and not vmm.handles and not vmm.mapped
+
+
+@pytest.mark.parametrize("k", [0, 1, 3])
+@pytest.mark.parametrize("keep", [False, True])
+def test_shrink_that_fails_half_way_keeps_books_and_mappings_in_step(vmm, k, keep):
+    """The driver refuses the unmap of range k: ranges before k are unmapped (and released), the rest stay mapped,
+    the pool still says grown while the live limit is already down; a second ekv_shrink finishes the job."""
+    pool = _create(num_layers=4, flags=ekv.EKV_START_GROWN)
+    flags = ekv.EKV_KEEP_PHYSICAL if keep else 0
+    vmm.fail_unmap_at = k
+    with pytest.raises(ekv.EkvError) as e:
+        ekv.ekv_shrink(pool, flags=flags, host_only=True)
+    assert e.value.status == ekv.Status.ERR_CUDA and f"layer {k}" in str(e.value)
+    info = ekv.ekv_pool_info(pool)
+    assert info.grown and info.live_blocks == info.base_blocks     # no kernel may reach the elastic ids any more
+    assert len(vmm.mapped) == 4 + (4 - k)                           # base mappings + elastic ones from range k on
+    assert len(vmm.handles) == (8 if keep else 8 - k)
+    with pytest.raises(ekv.EkvError) as e:                         # still "grown": a grow is refused, not stacked on top
+        ekv.ekv_grow(pool, host_only=True)
+    assert e.value.status == ekv.Status.ERR_STATE
+    ekv.ekv_shrink(pool, flags=flags, host_only=True)              # the retry touches only what is left
+    info = ekv.ekv_pool_info(pool)
+    assert not info.grown and len(vmm.mapped) == 4 and len(vmm.handles) == (8 if keep else 4)
+    assert bool(info.physical_held) == keep
+    ekv.ekv_grow(pool, host_only=True)                             # and the pool is fully usable afterwards
+    assert ekv.ekv_pool_info(pool).live_blocks == 192 and len(vmm.mapped) == 8
+    ekv.ekv_pool_destroy(pool)
+    assert not vmm.reserved and not vmm.handles and not vmm.mapped
+
+
+def test_live_limit_follows_every_toggle(vmm):
+    pool = _create(num_layers=2)
+    assert ekv.ekv_pool_info(pool).live_blocks == 128
+    ekv.ekv_grow(pool, host_only=True)
+    assert ekv.ekv_pool_info(pool).live_blocks == 192
+    ekv.ekv_shrink(pool, flags=ekv.EKV_KEEP_PHYSICAL, host_only=True)
+    assert ekv.ekv_pool_info(pool).live_blocks == 128
+    vmm.fail_map_at = 1                                            # a grow that fails leaves the limit where it was
+    with pytest.raises(ekv.EkvError):
+        ekv.ekv_grow(pool, host_only=True)
+    info = ekv.ekv_pool_info(pool)
+    assert info.live_blocks == 128 and not info.grown and len(vmm.mapped) == 2
+    ekv.ekv_pool_destroy(pool)
+
+
+def test_workspace_bytes_cover_every_smaller_shape(vmm):
+    """ekv_attn_workspace_bytes(max_batch, max_seq_len) promises room for EVERY call with B <= max_batch and a table
+    no wider than max_seq_len allows -- a shorter table can be cut into more key ranges than a longer one, so the
+    largest shape alone is not the bound.  Host-only pools plan for 148 SMs."""
+    for heads in ((32, 8), (64, 8), (8, 8)):
+        pool = _create(num_q_heads=heads[0], num_kv_heads=heads[1])
+        for max_batch, max_blocks in ((1, 8192), (4, 1024), (3, 785), (37, 300), (256, 512), (2, 17), (5, 2353)):
+            have = ekv.ekv_attn_workspace_bytes(pool, max_batch, max_blocks * 16)
+            worst = 0
+            for B in range(1, max_batch + 1):
+                step = max(1, max_blocks // 700)
+                for mb in list(range(1, max_blocks + 1, step)) + [max_blocks]:
+                    chunk, nsplit, need = ekv.ekv_attn_decode_plan(pool, B, mb)
+                    assert chunk % 64 == 0 and 64 <= chunk <= 2048 and (nsplit - 1) * chunk < mb * 16 <= nsplit * chunk
+                    worst = max(worst, need)
+            assert worst <= have, (heads, max_batch, max_blocks, worst, have)
+            assert have <= 2 * worst + 4096                        # a bound, not a blank cheque
+        ekv.ekv_pool_destroy(pool)
+    # the two shapes a review found short by a few KiB with the plan of the largest shape alone (32q/8kv, d128, 148 SMs)
+    pool = _create()
+    assert ekv.ekv_attn_decode_plan(pool, 1, 2353)[2] <= ekv.ekv_attn_workspace_bytes(pool, 1, 8192 * 16)
+    assert ekv.ekv_attn_decode_plan(pool, 3, 785)[2] <= ekv.ekv_attn_workspace_bytes(pool, 4, 1024 * 16)
+    ekv.ekv_pool_destroy(pool)
