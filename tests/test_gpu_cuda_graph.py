@@ -9,7 +9,9 @@ import pytest
 import torch
 
 import ekv_inputs as I
+import oracle
 import paper_2608_23658_b200 as ekv
+from helpers import assert_close, mirror_after_step
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -52,6 +54,16 @@ def test_captured_decode_and_prefill_steps_replay_across_toggles():
         step()                                     # eager warm-up: first-call set-up happens outside the capture
         torch.cuda.synchronize()
         eager = [o.clone() for o in outs] + [outp.clone()]
+        # the eager step against the oracle (every layer's decode of all six sequences, and the straddler's chunk);
+        # the replays below are then pinned to it bit for bit
+        for l in range(NL):
+            cache, ctab, clen = mirror_after_step(9, l, tables, lengths, range(B), s, k.cpu(), v.cpu())
+            want = oracle.attn_decode(cache, s.num_q_heads, s.num_kv_heads, 16, s.head_dim, q.cpu(), ctab, clen, scale)
+            assert_close(eager[l], want, f"eager decode, layer {l}")
+            if l == 0:
+                wantp = oracle.attn_prefill_chunk(cache, s.num_q_heads, s.num_kv_heads, 16, s.head_dim, qp.cpu(), ctab[2:3],
+                                                  cu, clen[2:3], scale)
+                assert_close(eager[NL], wantp, "eager prefill chunk of the straddler")
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             step()

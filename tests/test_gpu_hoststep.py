@@ -6,6 +6,8 @@ import pytest
 import torch
 
 import ekv_inputs as I
+import oracle
+from helpers import assert_close, bf16_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -54,6 +56,18 @@ def test_hoststep_matches_resident_calls_bitwise(depth):
             for t in range(steps):
                 assert torch.equal(host_in[t]["out"].view(torch.int16), want[t].view(torch.int16)), f"step {t}"
             assert torch.equal(pool.layer_tensor(0).view(torch.int16), ref.layer_tensor(0).view(torch.int16))
+            # the last step against the oracle, on a host mirror built from the seeded fill plus every step's rows
+            # (scattered by the oracle): all earlier writes of the pipeline must have landed for this to agree
+            final = lengths0 + steps
+            cache, ctab, _ = I.compact_host_cache(91, 0, tables, final, range(B), s)
+            cache = bf16_bits(cache).copy()
+            for t in range(steps):
+                slots = I.last_token_slots(lengths0 + t + 1, ctab, s.block_size)
+                assert oracle.write_kv(cache, cache.size // s.block_elems, s.num_kv_heads, s.block_size, s.head_dim,
+                                       host_in[t]["k"], host_in[t]["v"], slots) == 0
+            want_last = oracle.attn_decode(cache, s.num_q_heads, s.num_kv_heads, s.block_size, s.head_dim, host_in[-1]["q"],
+                                           ctab, final, scale)
+            assert_close(host_in[-1]["out"], want_last, "last pipelined step")
             # pure decode (no write) and a smaller batch reuse the same object
             hb = host_in[-1]
             out2 = torch.empty_like(hb["out"]).pin_memory()

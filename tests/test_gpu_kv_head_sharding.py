@@ -9,7 +9,9 @@ import pytest
 import torch
 
 import ekv_inputs as I
+import oracle
 import paper_2608_23658_b200 as ekv
+from helpers import assert_close, empty_cache, place_sequence
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -44,6 +46,15 @@ def test_sharded_pools_reproduce_the_head_slices_of_the_full_pool(tp):
     c = 260
     Qp = I.normal_bf16(19, 3, 0, c * 32 * 128).view(c, 32, 128)
     dec_full, pre_full = _run(full, K, V, Q, Qp, lengths, tables, 2, c)
+    # the full pool against the oracle; the shards are then compared with the full pool
+    host = empty_cache(int(tables.max()) + 1, full)
+    for b in range(len(lengths)):
+        place_sequence(host, full, tables[b], K[b], V[b])
+    scale = 1 / math.sqrt(128)
+    assert_close(dec_full, oracle.attn_decode(host, 32, 8, 16, 128, Q, tables, lengths, scale), "full-pool decode")
+    cu = np.array([0, c], dtype=np.int32)
+    assert_close(pre_full, oracle.attn_prefill_chunk(host, 32, 8, 16, 128, Qp, tables[2:3], cu, lengths[2:3], scale),
+                 "full-pool prefill chunk")
     hk, hq = 8 // tp, 32 // tp
     for rank in range(tp):
         shard = I.Shape(hq, hk, 128)
@@ -56,3 +67,9 @@ def test_sharded_pools_reproduce_the_head_slices_of_the_full_pool(tp):
         # decode: the split plan depends on B*Hkv, so the summation order may differ: tolerance
         d = (dec - dec_full[:, rank * hq:(rank + 1) * hq]).abs()
         assert d.max().item() <= 2e-2 and d.mean().item() <= 2e-3
+        # and the shard on its own against the oracle run on the shard's heads only (a narrower cache)
+        hosts = empty_cache(int(tables.max()) + 1, shard)
+        for b in range(len(lengths)):
+            place_sequence(hosts, shard, tables[b], Ks[b], Vs[b])
+        want = oracle.attn_decode(hosts, hq, hk, 16, 128, Q[:, rank * hq:(rank + 1) * hq].contiguous(), tables, lengths, scale)
+        assert_close(dec, want, f"decode of shard {rank}/{tp}")

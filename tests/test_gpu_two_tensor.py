@@ -7,7 +7,9 @@ import pytest
 import torch
 
 import ekv_inputs as I
+import oracle
 import paper_2608_23658_b200 as ekv
+from helpers import assert_close, mirror_after_step
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -34,6 +36,12 @@ def test_two_tensor_decode_matches_single_range_bitwise_and_reports_its_cost():
         two = torch.empty_like(q)
         ekv.ekv_attn_decode_two_tensor(pool.handle, 0, second, q, two, d_tables, d_lens, scale, ws)
         assert torch.equal(single, two)
+        # the oracle on a sample of the sequences (longest, shortest, and the one with the most elastic blocks), so that
+        # "same bits as the single-range kernel" also means "right"
+        sample = sorted({int(lengths.argmax()), int(lengths.argmin()), int((tables >= base).sum(1).argmax()), 0})
+        cache, ctab, clen = mirror_after_step(23, 0, tables, lengths, sample, s)
+        want = oracle.attn_decode(cache, s.num_q_heads, s.num_kv_heads, 16, s.head_dim, q[sample].cpu(), ctab, clen, scale)
+        assert_close(two[sample], want, "two-tensor decode")
         pool.shrink()                                                          # the two-tensor kernel needs no elastic range
         two2 = torch.empty_like(q)
         ekv.ekv_attn_decode_two_tensor(pool.handle, 0, second, q, two2, d_tables, d_lens, scale, ws)

@@ -1,8 +1,11 @@
 """The multi-GPU form of the benchmark is N independent replicas (the path has no exchange step).
 World-size-2 check on CPU (gloo) of the only cross-rank logic there is: the job's time is the MAX over
-ranks, the value is the whole-job aggregate, and the reference arm runs on rank 0 alone."""
+ranks, the value is the whole-job aggregate, and the reference arm runs on rank 0 alone; plus the launch
+path itself: `bench.py --gpus 2` started plainly starts two ranks, which rendezvous and report n_gpus 2."""
+import json
 import os
 import socket
+import subprocess
 import sys
 
 import torch
@@ -59,3 +62,26 @@ def test_reference_arm_runs_on_rank_zero_only(monkeypatch, capsys):
     monkeypatch.setenv("RANK", "1")
     assert bench.run_reference(Args) is None
     assert capsys.readouterr().out == ""
+
+
+def test_bench_started_plainly_with_gpus_2_starts_two_ranks_itself():
+    """No torchrun: bench.py spawns the ranks (RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* as torchrun would set them).
+    The GPU step is replaced by a host sleep of (rank + 1) x 20 ms (test hook --stub-ms) and the group runs on gloo;
+    the reported time must be the slow rank's, the value the aggregate of both replicas."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "4", "--stub-ms", "20"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout                                      # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["steps"] == 4 and line["scaling"] == "weak"
+    assert line["ms_per_step"] >= 40.0 > line["local_ms_rank0"] / 4      # the max over ranks, not rank 0's own time
+    assert abs(line["value"] - 2 * 1.0 * 4 / (line["ms_per_step"] * 4 * 1e-3)) < 0.05 * line["value"]
+
+
+def test_bench_refuses_a_world_size_that_contradicts_gpus():
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(_free_port()))
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--steps", "1", "--stub-ms", "1"],
+                       env=env, capture_output=True, text=True, timeout=120)
+    assert r.returncode != 0 and "--gpus 4" in r.stderr

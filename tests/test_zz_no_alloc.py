@@ -1,16 +1,20 @@
 """ekv_attn_decode_static_scratch: decode attention for callers that cannot allocate device memory
 (an engine whose free memory all went to the KV pool, a host without an allocator, a path where
 cudaMalloc must not be entered).  The scratch of the split pass is a fixed array inside the library;
-this file checks, through the C ABI, that the call gives what ekv_attn_decode gives, on two calls in
-a row (the array is shared and keeps the previous call's contents), and that a shape whose scratch
-need exceeds the array is refused.  It is collected last on purpose."""
+this file checks, through the C ABI, that the call gives what ekv_attn_decode gives -- the same bits:
+both run the same plan and kernels and differ only in where the partials live -- on two calls in a row
+(the array is shared and keeps the previous call's contents), that this is also what the CPU oracle
+computes, that the device's free memory and torch's own allocator do not move across a call, and that a
+shape whose scratch need exceeds the array is refused.  It is collected last on purpose."""
 import math
 
 import pytest
 import torch
 
 import ekv_inputs as I
+import oracle
 import paper_2608_23658_b200 as ekv
+from helpers import assert_close, mirror_after_step
 
 pytestmark = pytest.mark.gpu
 
@@ -25,13 +29,10 @@ def _workload(pool, shape, lengths, seed):
     I.fill_pool_layer_(pool.layer_tensor(0), seed)
     q = I.normal_bf16(seed, 3, 0, len(lengths) * shape.num_q_heads * shape.head_dim).view(
         len(lengths), shape.num_q_heads, shape.head_dim)
-    return q.to(DEV), tables.to(DEV), lengths.to(torch.int32).to(DEV)
-
-
-def _close(a, b):
-    d = (a.float() - b.float()).abs()
-    assert torch.isfinite(a.float()).all()
-    assert d.max().item() <= MAX_ABS and d.mean().item() <= MEAN_ABS, (d.max().item(), d.mean().item())
+    cache, ctab, clen = mirror_after_step(seed, 0, tables, lengths, range(len(lengths)), shape)
+    want = oracle.attn_decode(cache, shape.num_q_heads, shape.num_kv_heads, shape.block_size, shape.head_dim, q, ctab, clen,
+                              1 / math.sqrt(shape.head_dim))
+    return q.to(DEV), tables.to(DEV), lengths.to(torch.int32).to(DEV), want
 
 
 def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
@@ -42,15 +43,20 @@ def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
     try:
         # two different shapes back to back: the second call finds the first call's partials in the array
         for lengths, seed in (([3000, 17, 1, 2048, 999, 4100], 5), ([64, 700], 6)):
-            q, tables, lens = _workload(pool, shape, lengths, seed)
+            q, tables, lens, oracle_out = _workload(pool, shape, lengths, seed)
             want = pool.attn_decode(0, q, tables, lens, scale)              # existing entry point
             got = torch.full_like(q, float("nan"))
             ekv.ekv_attn_decode_static_scratch(pool.handle, 0, q, got, tables, lens, scale)
-            _close(got, want)
             again = torch.full_like(q, float("nan"))
-            ekv.ekv_attn_decode_static_scratch(pool.handle, 0, q, again, tables, lens, scale)
-            _close(again, want)
             torch.cuda.synchronize()
+            # the first call on the device has resolved the array's address; from here on a call must not
+            # move the device's free memory nor enter torch's allocator
+            free0, torch0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+            ekv.ekv_attn_decode_static_scratch(pool.handle, 0, q, again, tables, lens, scale)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == torch0
+            assert torch.equal(got, want) and torch.equal(again, want)
+            assert_close(got, oracle_out, "static-scratch decode", MAX_ABS, MEAN_ABS)
         assert pool.poll_status() == ekv.Status.OK
     finally:
         pool.close()
