@@ -7,7 +7,9 @@ One "step" = one pass of the hot path over one batch of the Llama-3-8B-shaped de
 (benchmark configs[1]): ekv_write_kv of the 256 new K/V rows through the slot mapping, then
 ekv_attn_decode (split pass + combine pass) of 256 sequences with context lengths U[1024, 8192]
 whose blocks are randomly permuted over the pool.  value = algorithmic bytes of the step / time.
-Multi-GPU runs are independent replicas (one pool per rank, no collective on the data path).
+Multi-GPU runs are independent replicas (one pool per rank, no collective on the data path): under
+torchrun the ranks come from the environment; started plainly with --gpus N > 1 this script starts the
+N ranks itself.
 
 The JSON line also carries: roofline (decode kernels, timed live with CUDA events), e2e (same
 step through host buffers), cpu_baseline (the CPU oracle on this machine's host cores), and two side
@@ -36,9 +38,10 @@ METRIC = "decode-attn HBM GB/s (% peak); prefill-chunk TFLOP/s (% peak); grow/sh
 UNIT = "GB/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes (read + write) per algorithmic byte of the decode split kernel, from the ncu capture
-# summarised in profiles/decode_split_c2_batch32.md (a 32-sequence slice of the same workload; the
-# traffic is proportional to the KV bytes read, so it is scaled to the full launch by that ratio).
+# DRAM bytes (read + write) per algorithmic byte of the decode split kernel: dram__bytes_read.sum +
+# dram__bytes_write.sum of one ncu capture of a 32-sequence slice of this workload (623.65 MB read, 4.77 MB
+# written, 622.92 MB algorithmic).  The traffic is proportional to the KV bytes read, so the full launch is
+# that ratio times its algorithmic bytes.  The capture has to be retaken whenever decode_split_kernel changes.
 DECODE_SPLIT_DRAM_TRAFFIC_RATIO = (623.649792 + 4.772352) / 622.920860
 
 
@@ -62,7 +65,12 @@ class ClockSampler:
     NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+        # nvidia-smi numbers the GPUs of the machine, CUDA the visible ones: address the device by its UUID
+        try:
+            self.index = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+        except Exception:
+            self.index = str(index)
+        self.rows, self.proc = [], None
 
     def __enter__(self):
         try:
@@ -231,9 +239,24 @@ def timed_loop(fn, steps, device, dist):
 # ----------------------------------------------------------------------------- side measurements
 
 
-def measure_prefill(device, peaks, reps=3, prompt_len=None, chunks=None):
+def _time_reps(fn, device, reps):
+    """ms of `reps` separately timed runs of fn (CUDA events on the current stream), after one warm-up run."""
+    fn()
+    torch.cuda.synchronize(device)
+    ts = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize(device)
+        ts.append(e0.elapsed_time(e1))
+    return ts
+
+
+def measure_prefill(device, peaks, reps=5, prompt_len=None, chunks=None):
     """Prefill-chunk TFLOP/s on the configs[2] prompt: 32768 tokens as four 8192-token chunks over
-    cached prefixes 0/8k/16k/24k, and as one 32768-token chunk."""
+    cached prefixes 0/8k/16k/24k, and as one 32768-token chunk.  Median of `reps` runs, with min and max."""
     import paper_2608_23658_b200 as ekv
     cfg, s = I.C3, I.C3.shape
     Lp = prompt_len or cfg.prompt_len
@@ -259,25 +282,48 @@ def measure_prefill(device, peaks, reps=3, prompt_len=None, chunks=None):
             def run():
                 for (qq, oo, cud, cuh, sl) in calls:
                     pool.attn_prefill_chunk(0, qq, d_table, cud, cuh, sl, scale, out=oo)
-            run()
-            torch.cuda.synchronize(device)
-            best = float("inf")
-            for _ in range(reps):
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                run()
-                e1.record()
-                torch.cuda.synchronize(device)
-                best = min(best, e0.elapsed_time(e1))
+            ts = _time_reps(run, device, reps)
+            med = statistics.median(ts)
             flops = sum(I.prefill_flops(chunk, start, s) for start in range(0, Lp, chunk))
-            tf = flops / (best * 1e-3) / 1e12
-            res[f"chunk_{chunk}"] = {"ms": round(best, 3), "tflops": round(tf, 1),
+            tf = flops / (med * 1e-3) / 1e12
+            res[f"chunk_{chunk}"] = {"ms": round(med, 3), "ms_min": round(min(ts), 3), "ms_max": round(max(ts), 3),
+                                     "tflops": round(tf, 1), "launches": len(calls),
                                      "frac_of_measured_bf16": round(tf / peaks["bf16_tflops"], 4),
                                      "frac_of_nominal_2250": round(tf / 2250.0, 4)}
-        res["workload"] = "c3 prompt 32768 tokens, 32/8 heads d128, causal-exact FLOPs of both contractions"
+        res["workload"] = f"c3 prompt {Lp} tokens, 32/8 heads d128, causal-exact FLOPs of both contractions, median of {reps}"
         return res
     finally:
         pool.close()
+
+
+def measure_prefill_short(device, peaks, reps=5):
+    """The same 32768 query tokens as many short prompts without a cached prefix, one call per batch:
+    64 prompts of 512 tokens and 256 prompts of 128 tokens (what a batch of fresh short requests looks like)."""
+    import paper_2608_23658_b200 as ekv
+    cfg, s = I.C3, I.C3.shape
+    T = 32768
+    res = {}
+    for R, c in ((64, 512), (256, 128)):
+        lengths = torch.full((R,), c, dtype=torch.int64)
+        pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim,
+                        base_blocks=T // s.block_size + 64, device=device.index or 0)
+        try:
+            tables, _ = I.assign_blocks(cfg.seed, 15, lengths, s.block_size, pool.info.live_blocks)
+            I.fill_pool_layer_(pool.layer_tensor(0), cfg.seed)
+            q = I.normal_bf16(cfg.seed, 6, 0, T * s.num_q_heads * s.head_dim, device=device).view(T, s.num_q_heads, s.head_dim)
+            out = torch.empty_like(q)
+            cu = torch.arange(0, T + 1, c, dtype=torch.int32)
+            d_cu, d_tables, d_lens = cu.to(device), tables.to(device), lengths.to(torch.int32).to(device)
+            scale = 1.0 / math.sqrt(s.head_dim)
+            ts = _time_reps(lambda: pool.attn_prefill_chunk(0, q, d_tables, d_cu, cu, d_lens, scale, out=out), device, reps)
+            med = statistics.median(ts)
+            tf = R * I.prefill_flops(c, 0, s) / (med * 1e-3) / 1e12
+            res[f"{R}x{c}"] = {"ms": round(med, 4), "ms_min": round(min(ts), 4), "tflops": round(tf, 1),
+                               "frac_of_measured_bf16": round(tf / peaks["bf16_tflops"], 4)}
+        finally:
+            pool.close()
+    res["workload"] = "32768 query tokens as R prompts of c tokens, no cached prefix, one call, 32/8 heads d128"
+    return res
 
 
 def measure_mixed_step(device, peaks, reps=5):
@@ -467,20 +513,39 @@ def measure_write_kv(device, peaks):
     return res
 
 
-def measure_decode_long_context(device, peaks, reps=5):
+def measure_decode_long_context(device, peaks, reps=5, hbm_filling=False):
     """Decode attention on the configs[3] batch (64 sequences, 64q/8kv heads, contexts U[32768,131072], 21.3 GB of KV
-    per launch) in a pool just large enough for it."""
+    per launch).  hbm_filling=False: a pool just large enough for the batch.  hbm_filling=True: the pool configs[3]
+    describes -- min(140 GiB, free memory - 10 GiB), 16 % of its block ids elastic, the batch's blocks drawn by a
+    uniform permutation over ALL of it (only the blocks the batch touches are filled) -- so that the table walk
+    jumps over the whole of HBM and the translation reach of the memory system is part of what is timed."""
     import paper_2608_23658_b200 as ekv
     cfg, s = I.C4, I.C4.shape
     lengths = I.decode_lengths(cfg)
     need = int(I.blocks_for(lengths, s.block_size).sum())
-    elastic = int(need * 1.02 * cfg.elastic_fraction)
+    if hbm_filling:
+        free, _ = torch.cuda.mem_get_info(device)
+        total = min(140 << 30, free - (10 << 30)) // s.block_bytes
+        if total < need * 1.02:
+            return {"skipped": f"only {free / 2**30:.1f} GiB free: the pool cannot hold the draw"}
+    else:
+        total = int(need * 1.02)
+    elastic = int(total * cfg.elastic_fraction)
     pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim,
-                    base_blocks=int(need * 1.02) - elastic, elastic_blocks=elastic, start_grown=True, device=device.index or 0)
+                    base_blocks=total - elastic, elastic_blocks=elastic, start_grown=True, device=device.index or 0)
     try:
         live = pool.info.live_blocks
         tables, _ = I.assign_blocks(cfg.seed, 12, lengths, s.block_size, live)
-        I.fill_pool_layer_(pool.layer_tensor(0), cfg.seed, chunk=1 << 26)
+        view = pool.layer_tensor(0)
+        if hbm_filling:
+            ids_sorted = torch.sort(tables[tables >= 0].long()).values.to(device)
+            ar = torch.arange(s.block_elems, device=device)[None]
+            for o in range(0, len(ids_sorted), 4096):
+                idx = ids_sorted[o:o + 4096]
+                vals = I.normal_bf16_at(cfg.seed, I.KV_STREAM, (idx[:, None] * s.block_elems + ar).reshape(-1))
+                view[idx] = vals.view(len(idx), 2, s.num_kv_heads, s.block_size, s.head_dim)
+        else:
+            I.fill_pool_layer_(view, cfg.seed, chunk=1 << 26)
         B = len(lengths)
         q = I.normal_bf16(cfg.seed, 3, 0, B * s.num_q_heads * s.head_dim, device=device).view(B, s.num_q_heads, s.head_dim)
         d_tables, d_lens = tables.to(device), lengths.to(torch.int32).to(device)
@@ -500,8 +565,9 @@ def measure_decode_long_context(device, peaks, reps=5):
         gbs = nbytes / ms / 1e6
         return {"ms": round(ms, 3), "gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
                 "frac_of_nominal_8000": round(gbs / 8000.0, 4), "algorithmic_bytes": nbytes,
-                "elastic_fraction_of_blocks": round(elastic / live, 3),
-                "workload": "c4 decode: 64 seqs, 64q/8kv heads d128, contexts U[32768,131072]"}
+                "pool_gib": round(live * s.block_bytes / 2**30, 1), "elastic_fraction_of_blocks": round(elastic / live, 3),
+                "workload": "c4 decode: 64 seqs, 64q/8kv heads d128, contexts U[32768,131072], " +
+                            ("HBM-filling pool, blocks scattered over all of it" if hbm_filling else "pool just large enough")}
     finally:
         pool.close()
 
@@ -509,15 +575,24 @@ def measure_decode_long_context(device, peaks, reps=5):
 # ----------------------------------------------------------------------------- CPU oracle legs
 
 
-def oracle_decode_sample(cfg, max_seqs=24):
-    """Times the CPU oracle, as it stands, on a bounded sample of the decode workload."""
+def _generator_device():
+    """Where the seeded value generator runs when a host mirror is built: the bits are the same on every torch
+    device (integer arithmetic and one IEEE multiply), a GPU just produces gigabytes of them in seconds."""
+    return "cuda" if torch.cuda.is_available() else "cpu"
+
+
+def oracle_decode_sample(cfg, max_seqs=None):
+    """Times the CPU oracle, as it stands, on the decode workload: all of its sequences when the host mirror can be
+    generated quickly (a GPU is present), otherwise the first 24."""
     import oracle
     s = cfg.shape
     lengths = I.decode_lengths(cfg)
+    if max_seqs is None:
+        max_seqs = len(lengths) if _generator_device() == "cuda" else 24
     need = int(I.blocks_for(lengths, s.block_size).sum())
     tables, _ = I.assign_blocks(cfg.seed, 12, lengths, s.block_size, int(need * 1.1) + 64)
     ids = list(range(min(max_seqs, len(lengths))))
-    cache, ctab, clen = I.compact_host_cache(cfg.seed, 0, tables, lengths, ids, s)
+    cache, ctab, clen = I.compact_host_cache(cfg.seed, 0, tables, lengths, ids, s, device=_generator_device())
     q = I.normal_bf16(cfg.seed, 3, 0, len(lengths) * s.num_q_heads * s.head_dim).view(len(lengths), s.num_q_heads, s.head_dim)
     qs = q[ids].contiguous()
     scale = 1.0 / math.sqrt(s.head_dim)
@@ -528,8 +603,34 @@ def oracle_decode_sample(cfg, max_seqs=24):
         t0 = time.perf_counter()
         oracle.attn_decode(cache, s.num_q_heads, s.num_kv_heads, s.block_size, s.head_dim, qs, ctab, clen, scale)
         return time.perf_counter() - t0
-    return one, nbytes, f"{len(ids)} of {len(lengths)} sequences of the workload ({int(clen.sum())} cached tokens, all heads)", \
+    which = "all" if len(ids) == len(lengths) else f"{len(ids)} of"
+    return one, nbytes, f"{which} {len(lengths)} sequences of the workload ({int(clen.sum())} cached tokens, all heads)", \
         oracle.threads()
+
+
+def oracle_prefill_sample(rows_per_chunk=16):
+    """The CPU oracle on a row sample of the configs[2] prompt (32768 tokens, one request, no prefix): first and
+    last row of every 8192-token chunk plus rows spread evenly, all 32 heads.  Returns a dict with its GFLOP/s
+    (causal-exact FLOPs of the sampled rows only)."""
+    import oracle
+    cfg, s = I.C3, I.C3.shape
+    Lp = cfg.prompt_len
+    table, _ = I.assign_blocks(cfg.seed, 13, torch.tensor([Lp]), s.block_size, Lp // s.block_size + 64)
+    cache, ctab, clen = I.compact_host_cache(cfg.seed, 0, table, torch.tensor([Lp]), [0], s, device=_generator_device())
+    q = I.normal_bf16(cfg.seed, 6, 0, Lp * s.num_q_heads * s.head_dim).view(Lp, s.num_q_heads, s.head_dim)
+    rows = set()
+    for start in range(0, Lp, 8192):
+        rows |= {start, start + 8191} | {start + (8192 * k) // rows_per_chunk for k in range(rows_per_chunk)}
+    rows = sorted(rows)
+    cu = torch.tensor([0, Lp], dtype=torch.int32)
+    scale = 1.0 / math.sqrt(s.head_dim)
+    t0 = time.perf_counter()
+    oracle.attn_prefill_chunk(cache, s.num_q_heads, s.num_kv_heads, s.block_size, s.head_dim, q, ctab, cu, clen, scale,
+                              rows=torch.tensor(rows, dtype=torch.int32))
+    dt = time.perf_counter() - t0
+    flops = 4 * s.head_dim * s.num_q_heads * sum(r + 1 for r in rows)
+    return {"gflops": round(flops / dt / 1e9, 2), "seconds": round(dt, 3), "cores": oracle.threads(),
+            "sample": f"{len(rows)} of {Lp} query rows of the c3 prompt (chunk borders + evenly spread), all heads"}
 
 
 def run_reference(args):
@@ -548,7 +649,7 @@ def run_reference(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(1e3 * total / args.steps, 3),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": cfg.name, "batch": cfg.decode.batch, "heads": "32q/8kv", "head_dim": 128, "block_size": 16,
-                       "step": "oracle attn_decode on a sample of the workload's sequences", "sample": sample},
+                       "step": "oracle attn_decode (the write of the step's 256 rows is not timed)", "sample": sample},
             "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -558,7 +659,52 @@ def run_reference(args):
 # ----------------------------------------------------------------------------- main
 
 
-def main():
+def _free_port():
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_ranks(n: int, argv) -> int:
+    """`bench.py --gpus N` started plainly (no torchrun): start the N ranks here, one process per GPU, each with
+    the environment torchrun would give it (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR, MASTER_PORT).  Rank 0's
+    stdout is this process's stdout, so its JSON line is the job's.  Returns the worst exit code."""
+    port = _free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *argv], env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    return max(abs(p.wait()) for p in procs)
+
+
+def run_stub(args, rank, world):
+    """Test hook (--stub-ms): the launch, rendezvous, timing and reporting logic of a replica run with the GPU step
+    replaced by a host sleep of (rank + 1) x stub_ms and the process group on gloo, so that the multi-rank path can
+    be exercised on a machine without GPUs."""
+    import torch.distributed as dist
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    cpu = torch.device("cpu")
+    dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(args.stub_ms * (rank + 1) * 1e-3)
+    local_ms = (time.perf_counter() - t0) * 1e3
+    ms = max_over_ranks(local_ms, dist, cpu)
+    dist.barrier()
+    if rank == 0:
+        step_bytes = 1_000_000_000
+        print(json.dumps({"metric": METRIC, "value": round(whole_job_gbs(step_bytes, args.steps, ms, world), 3), "unit": UNIT,
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4),
+                          "scaling": "weak", "data": "stub", "local_ms_rank0": round(local_ms, 3),
+                          "config": {"workload": "stub step (host sleep), replicas only"}}), flush=True)
+    dist.destroy_process_group()
+
+
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=500)
@@ -569,18 +715,29 @@ def main():
     ap.add_argument("--prefill-only", type=int, default=0, metavar="PROMPT_LEN",
                     help="profiling aid: run only the prefill-chunk measurement on a prompt of this length "
                          "(one-shot and in 4 chunks) and print its JSON")
+    ap.add_argument("--prefill-short-only", action="store_true",
+                    help="profiling aid: run only the many-short-prompts prefill measurement and print its JSON")
     ap.add_argument("--write-kv-only", action="store_true",
                     help="profiling aid: run only the ekv_write_kv measurement (8192 and 32768 tokens) and print its JSON")
-    args = ap.parse_args()
+    ap.add_argument("--stub-ms", type=float, default=0.0,
+                    help="test hook: replace the GPU step by a host sleep of (rank+1) x this many ms, ranks on gloo")
+    args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3)
 
     if args.impl == "reference":
         run_reference(args)
-        return
+        return 0
 
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        return spawn_ranks(args.gpus, argv)
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if args.stub_ms > 0:
+        run_stub(args, rank, world)
+        return 0
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device; the ekv path has no CPU fallback (use --impl reference for the oracle)")
     device = torch.device("cuda", local_rank)
@@ -594,11 +751,14 @@ def main():
     peaks, peaks_kind = measured_peaks()
     if args.prefill_only:
         n = args.prefill_only
-        print(json.dumps({"prefill": measure_prefill(device, peaks, reps=2, prompt_len=n, chunks=(n // 4, n))}), flush=True)
-        return
+        print(json.dumps({"prefill": measure_prefill(device, peaks, reps=3, prompt_len=n, chunks=(n // 4, n))}), flush=True)
+        return 0
+    if args.prefill_short_only:
+        print(json.dumps({"prefill_short": measure_prefill_short(device, peaks, reps=3)}), flush=True)
+        return 0
     if args.write_kv_only:
         print(json.dumps({"write_kv": measure_write_kv(device, peaks)}), flush=True)
-        return
+        return 0
     cfg = I.C2
     wl = DecodeWorkload(cfg, device, args.batch)
     assert wl.decode_bytes > 200e6 or args.batch, "working set must exceed L2"
@@ -650,6 +810,7 @@ def main():
     e2e_value = whole_job_gbs(step_bytes, args.steps, ms_e2e, world)
     achieved = wl.decode_bytes / (decode_ms * 1e-3) / 1e9
     h2d, d2h = wl.e2e_bytes()
+    nsplit = wl.ekv.ekv_attn_decode_plan(wl.pool.handle, wl.B, int(wl.tables.shape[1]))[1]
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
@@ -658,28 +819,41 @@ def main():
                    "context_tokens": int(wl.lengths.sum()), "step": "ekv_write_kv + ekv_attn_decode (split + combine)",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2 (%.2f GB of KV per step)" % (wl.decode_bytes / 1e9)},
-        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel<128, false> + decode_combine_kernel<128>",
-                     "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": round(achieved / peaks["hbm_gbs"], 4), "peak_kind": f"{peaks_kind} copy bandwidth",
-                     "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": int(DECODE_SPLIT_DRAM_TRAFFIC_RATIO * wl.decode_bytes),
-                     "algorithmic_bytes_per_launch": wl.decode_bytes, "launch_ms": round(decode_ms, 4),
-                     "write_kv_ms": round(write_ms, 4)},
-        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": round(ms_e2e / args.steps, 4)},
-        "gpu_launches": 3 * args.steps,
+        "gpu_launches": (2 + (1 if nsplit > 1 else 0)) * args.steps,
         "clocks": clocks,
     }
+    roofline = {"bound": "hbm", "kernel": "decode_split_kernel<128, false> + decode_combine_kernel<128>",
+                "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": round(achieved / peaks["hbm_gbs"], 4), "peak_kind": f"{peaks_kind} copy bandwidth",
+                "frac_of_nominal_8000": round(achieved / 8000.0, 4), "traffic": int(DECODE_SPLIT_DRAM_TRAFFIC_RATIO * wl.decode_bytes),
+                "algorithmic_bytes_per_launch": wl.decode_bytes, "launch_ms": round(decode_ms, 4),
+                "write_kv_ms": round(write_ms, 4)}
+    e2e = {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "ms_per_step": round(ms_e2e / args.steps, 4)}
     wl.close()
     if rank == 0 and world == 1 and not args.no_extras:
-        torch.cuda.empty_cache()
-        line["prefill"] = measure_prefill(device, peaks)
-        torch.cuda.empty_cache()
-        line["mixed_step"] = measure_mixed_step(device, peaks)
+        # Side measurements of the other hot-path rows.  The bulky one (toggle) goes first and the compact ones
+        # last, so that the end of the line holds prefill, mixed step, long-context decode, write and the CPU baseline.
         torch.cuda.empty_cache()
         line["toggle"] = measure_toggle(device)
         torch.cuda.empty_cache()
+        line["decode_long_context_hbm_filling_pool"] = measure_decode_long_context(device, peaks, hbm_filling=True)
+        torch.cuda.empty_cache()
         line["decode_long_context"] = measure_decode_long_context(device, peaks)
         line["write_kv"] = measure_write_kv(device, peaks)
+        torch.cuda.empty_cache()
+        line["mixed_step"] = measure_mixed_step(device, peaks)
+        torch.cuda.empty_cache()
+        line["prefill_short"] = measure_prefill_short(device, peaks)
+        torch.cuda.empty_cache()
+        pf = measure_prefill(device, peaks)
+        line["prefill"] = pf
+        one_shot = pf["chunk_32768"]
+        line["roofline_prefill"] = {
+            "bound": "tensor", "kernel": "prefill_tc_kernel", "achieved": one_shot["tflops"], "peak": peaks["bf16_tflops"],
+            "unit": "TFLOP/s", "frac": one_shot["frac_of_measured_bf16"], "peak_kind": f"{peaks_kind} cuBLAS bf16 burst",
+            "launch_ms": one_shot["ms"], "workload": "c3 prompt, one 32768-token chunk",
+            "chunked_4x8192_tflops": pf["chunk_8192"]["tflops"], "traffic": None}
         one, nbytes, sample, cores = oracle_decode_sample(cfg)
         one()
         reps, t = 0, 0.0
@@ -687,12 +861,16 @@ def main():
             t += one()
             reps += 1
         line["cpu_baseline"] = {"value": round(nbytes * reps / t / 1e9, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"{sample}, {reps} passes"}
+                                "sample": f"{sample}, {reps} passes", "ms_per_pass": round(1e3 * t / reps, 1),
+                                "prefill_rows": oracle_prefill_sample()}
+    line["e2e"] = e2e
+    line["roofline"] = roofline
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+    return 0
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main())

@@ -236,17 +236,28 @@ def fill_pool_layer_(layer_view: torch.Tensor, seed: int, layer: int = 0, first_
         layer_view[b0:b1] = vals.view(b1 - b0, *layer_view.shape[1:])
 
 
-def host_blocks(seed: int, layer: int, block_ids, block_elems: int) -> torch.Tensor:
-    """CPU regeneration of the listed physical blocks of a fill_pool_layer_ pool: bf16 [n, block_elems]."""
+def host_blocks(seed: int, layer: int, block_ids, block_elems: int, device="cpu") -> torch.Tensor:
+    """Regeneration, in host memory, of the listed physical blocks of a fill_pool_layer_ pool: bf16 [n, block_elems].
+    The generator itself may run on another torch device (same bits everywhere); the result is returned on the CPU."""
     out = torch.empty(len(block_ids), block_elems, dtype=torch.bfloat16)
-    for i, n in enumerate(block_ids):
-        out[i] = normal_bf16(seed, KV_STREAM + layer, int(n) * block_elems, block_elems)
+    if torch.device(device).type == "cpu":
+        for i, n in enumerate(block_ids):
+            out[i] = normal_bf16(seed, KV_STREAM + layer, int(n) * block_elems, block_elems)
+        return out
+    ids = torch.as_tensor(block_ids, dtype=torch.int64, device=device)
+    ar = torch.arange(block_elems, dtype=torch.int64, device=device)[None]
+    per = max(1, (1 << 25) // block_elems)
+    for o in range(0, len(ids), per):
+        idx = (ids[o:o + per, None] * block_elems + ar).reshape(-1)
+        out[o:o + per] = normal_bf16_at(seed, KV_STREAM + layer, idx).view(-1, block_elems).cpu()
     return out
 
 
-def compact_host_cache(seed: int, layer: int, tables: torch.Tensor, lengths: torch.Tensor, seq_ids, shape: Shape):
+def compact_host_cache(seed: int, layer: int, tables: torch.Tensor, lengths: torch.Tensor, seq_ids, shape: Shape,
+                       device="cpu"):
     """Host mirror holding only the blocks of the listed sequences, renumbered 0..n-1.
-    Returns (cache bf16 [n*block_elems], compact tables int32 [len(seq_ids), width], lengths)."""
+    Returns (cache bf16 [n*block_elems], compact tables int32 [len(seq_ids), width], lengths).
+    `device`: where the value generator runs (the mirror always ends up in host memory)."""
     nb = blocks_for(lengths, shape.block_size)
     width = int(nb[list(seq_ids)].max())
     ctab = torch.full((len(seq_ids), width), -1, dtype=torch.int32)
@@ -255,7 +266,7 @@ def compact_host_cache(seed: int, layer: int, tables: torch.Tensor, lengths: tor
         n = int(nb[b])
         ctab[i, :n] = torch.arange(len(ids), len(ids) + n, dtype=torch.int32)
         ids += tables[b, :n].tolist()
-    cache = host_blocks(seed, layer, ids, shape.block_elems).view(-1)
+    cache = host_blocks(seed, layer, ids, shape.block_elems, device=device).view(-1)
     return cache, ctab, lengths[list(seq_ids)].clone()
 
 
