@@ -82,6 +82,13 @@ enum {
                                     until the next ekv_grow maps it again) */
     EKV_FUSED_RANGE = 1u << 2,   /* ekv_pool_create: ONE virtual range and two handles for all layers
                                     instead of one range and two handles per layer (see above) */
+    EKV_PREFILL_ONE_HEAD = 1u << 4, /* ekv_pool_create: ekv_attn_prefill_chunk on this pool always runs the
+                                    one-head-per-CTA tcgen05 kernel (normally chosen for head_dim 64, odd
+                                    query groups and batches of short chunks), so that it can be tested
+                                    and timed on any shape. */
+    EKV_PREFILL_TWO_HEAD = 1u << 5, /* ekv_pool_create: ekv_attn_prefill_chunk on this pool runs the two-head
+                                    tcgen05 kernel whenever the shape allows it (head_dim 128, even query
+                                    group, scale > 0), however short the chunks are. */
     EKV_PREFILL_WARP_MMA = 1u << 3 /* ekv_pool_create: ekv_attn_prefill_chunk on this pool always runs the
                                     warp-level (mma.sync) kernel, never a tcgen05 one.  Same results within
                                     the stated tolerance; exists so the two kernel families can be checked
@@ -96,7 +103,7 @@ typedef struct ekv_pool_desc {
     int32_t head_dim;       /* 64 or 128 */
     int32_t block_size;     /* 16 */
     int32_t dtype;          /* EKV_BF16 */
-    uint32_t flags;         /* EKV_START_GROWN | EKV_FUSED_RANGE | EKV_PREFILL_WARP_MMA */
+    uint32_t flags;         /* EKV_START_GROWN | EKV_FUSED_RANGE | EKV_PREFILL_* */
     int64_t base_blocks;    /* per layer, >= 1; rounded UP to whole granules */
     int64_t elastic_blocks; /* per layer, >= 0; rounded UP to whole granules */
 } ekv_pool_desc_t;

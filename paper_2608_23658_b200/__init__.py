@@ -5,7 +5,7 @@ every step of the path runs in the library's CUDA kernels.  There is no CPU fall
 library cannot be loaded, or no CUDA device exists, calls raise.
 """
 from ._binding import (  # noqa: F401
-    EKV_BF16, EKV_FUSED_RANGE, EKV_KEEP_PHYSICAL, EKV_PREFILL_WARP_MMA, EKV_START_GROWN, EkvError, PoolDesc, PoolInfo, VmmBackend, Status,
+    EKV_BF16, EKV_FUSED_RANGE, EKV_KEEP_PHYSICAL, EKV_PREFILL_ONE_HEAD, EKV_PREFILL_TWO_HEAD, EKV_PREFILL_WARP_MMA, EKV_START_GROWN, EkvError, PoolDesc, PoolInfo, VmmBackend, Status,
     EKV_STATIC_SCRATCH_BYTES, ekv_attn_decode, ekv_attn_decode_plan, ekv_attn_decode_static_scratch, ekv_attn_decode_two_tensor, ekv_attn_prefill_chunk, ekv_attn_workspace_bytes, ekv_grow, ekv_last_error, ekv_layer_ptr,
     ekv_poll_status, ekv_pool_create, ekv_pool_destroy, ekv_pool_info, ekv_set_vmm_backend, ekv_shrink,
     ekv_status_string, ekv_write_kv, library_path, load_library)

@@ -14,6 +14,8 @@ EKV_START_GROWN = 1
 EKV_KEEP_PHYSICAL = 2
 EKV_FUSED_RANGE = 4
 EKV_PREFILL_WARP_MMA = 8
+EKV_PREFILL_ONE_HEAD = 16
+EKV_PREFILL_TWO_HEAD = 32
 
 
 class Status(enum.IntEnum):

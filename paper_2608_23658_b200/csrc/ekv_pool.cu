@@ -316,7 +316,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
     if (d.num_layers < 1 || d.num_kv_heads < 1 || d.num_q_heads < d.num_kv_heads || d.num_q_heads % d.num_kv_heads != 0 ||
         d.num_q_heads / d.num_kv_heads > 8 || (d.head_dim != 64 && d.head_dim != 128) || d.block_size != 16 ||
         d.dtype != EKV_BF16 || d.base_blocks < 1 || d.elastic_blocks < 0 || d.device < 0 ||
-        (d.flags & ~(uint32_t)(EKV_START_GROWN | EKV_FUSED_RANGE | EKV_PREFILL_WARP_MMA)) != 0) {
+        (d.flags & ~(uint32_t)(EKV_START_GROWN | EKV_FUSED_RANGE | EKV_PREFILL_WARP_MMA | EKV_PREFILL_ONE_HEAD | EKV_PREFILL_TWO_HEAD)) != 0) {
         set_error("ekv_pool_create: unsupported geometry (layers %d, heads %d/%d, head_dim %d, block_size %d, dtype %d, "
                   "blocks %lld+%lld, flags 0x%x)",
                   d.num_layers, d.num_q_heads, d.num_kv_heads, d.head_dim, d.block_size, d.dtype, (long long)d.base_blocks,

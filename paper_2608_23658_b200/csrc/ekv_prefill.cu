@@ -1,10 +1,19 @@
 // ekv_attn_prefill_chunk: host entry point.  Validates, sizes the launch from the host copy of
 // cu_q_lens (no device synchronisation) and dispatches the kernel for the pool's head_dim.
 #include "ekv_internal.h"
+#ifndef EKV_SHORT_CHUNK_ROWS
+#define EKV_SHORT_CHUNK_ROWS 0
+#endif
 #include "ekv_prefill_mma.cuh"
 #include "ekv_prefill_tc.cuh"
+#include "ekv_prefill_tc1.cuh"
 
 using namespace ekv;
+
+// Mean chunk length (query rows per request of the call) below which the one-head kernel takes a head_dim 128 /
+// even-group call.  0 = never: measured on 64 x 512 and 256 x 128 fresh prompts the two-head kernel is the faster
+// of the two (348 vs 472 us, 279 vs 316 us), so the one-head kernel serves only the shapes the other cannot take.
+static constexpr int kShortChunkMeanRows = EKV_SHORT_CHUNK_ROWS;
 
 extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
                                                const int32_t *block_tables, int32_t max_blocks_per_seq,
@@ -23,13 +32,28 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
         set_error("ekv_attn_prefill_chunk: cu_q_lens[0] must be 0");
         return EKV_ERR_INVALID;
     }
-    // tcgen05 kernel: head_dim 128, query heads paired inside a kv group, positive scale.  Everything
-    // else (and every call on a pool created with EKV_PREFILL_WARP_MMA, which the tests use to check
-    // the two kernels against each other) takes the warp-level MMA kernel.
-    const bool force_mma = (pool->desc.flags & EKV_PREFILL_WARP_MMA) != 0;
+    // Three kernels (scale > 0 unless stated):
+    //   two-head tcgen05 kernel  head_dim 128, even query group, long chunks: a CTA owns the SM and every K/V tile feeds two heads
+    //   one-head tcgen05 kernel  head_dim 64, odd query groups, and batches of short chunks (two CTAs per SM hide each
+    //                            other's fixed cost); EKV_PREFILL_ONE_HEAD / EKV_PREFILL_TWO_HEAD override the choice between the two
+    //   warp-level MMA kernel    non-positive scales, and every call on a pool created with EKV_PREFILL_WARP_MMA (which
+    //                            the tests use to check the kernel families against each other)
+    // Only chunk lengths are known on the host (the prefixes live in seq_lens on the device), so "short" is judged by
+    // the mean chunk length of the call.
     const int group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
-    const bool use_tc = !force_mma && pool->desc.head_dim == 128 && group % 2 == 0 && scale > 0.f;
-    const int bm = use_tc ? tc::kBM : kPmBM;
+    const uint32_t pf = pool->desc.flags;
+    enum { K_TWO_HEAD, K_ONE_HEAD, K_WARP_MMA } kernel;
+    if ((pf & EKV_PREFILL_WARP_MMA) || !(scale > 0.f)) {
+        kernel = K_WARP_MMA;
+    } else if ((pf & EKV_PREFILL_ONE_HEAD) || pool->desc.head_dim != 128 || group % 2 != 0) {
+        kernel = K_ONE_HEAD;
+    } else if (pf & EKV_PREFILL_TWO_HEAD) {
+        kernel = K_TWO_HEAD;
+    } else {
+        const long long total_rows = cu_q_lens_host[R];
+        kernel = total_rows < (long long)kShortChunkMeanRows * R ? K_ONE_HEAD : K_TWO_HEAD;
+    }
+    const int bm = kernel == K_WARP_MMA ? kPmBM : tc::kBM;
     PrefillParams p;
     p.n_prefix = R <= kPrefixMax ? 1 : 0;
     long long q_tiles = 0;
@@ -63,7 +87,11 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     p.group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     p.R = R;
     p.scale_log2 = scale * 1.4426950408889634f;
-    if (use_tc) return tc::launch_prefill_tc(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
-    if (pool->desc.head_dim == 128) return launch_prefill_mma<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
-    return launch_prefill_mma<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
+    const bool d128 = pool->desc.head_dim == 128;
+    if (kernel == K_TWO_HEAD) return tc::launch_prefill_tc(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
+    if (kernel == K_ONE_HEAD)
+        return d128 ? tc1::launch_prefill_tc1<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream)
+                    : tc1::launch_prefill_tc1<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
+    return d128 ? launch_prefill_mma<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream)
+                : launch_prefill_mma<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
 }

@@ -17,14 +17,17 @@ class _RawCuda:
 
 class Pool:
     def __init__(self, *, num_q_heads, num_kv_heads, head_dim, base_blocks, elastic_blocks=0, num_layers=1,
-                 block_size=16, device=0, start_grown=False, fused_range=False, prefill_warp_mma=False):
+                 block_size=16, device=0, start_grown=False, fused_range=False, prefill_warp_mma=False,
+                 prefill_one_head=False, prefill_two_head=False):
         self.device = torch.device("cuda", device)
         torch.cuda.set_device(self.device)
         self.handle = B.ekv_pool_create(device=device, num_layers=num_layers, num_q_heads=num_q_heads,
                                         num_kv_heads=num_kv_heads, head_dim=head_dim, block_size=block_size,
                                         base_blocks=base_blocks, elastic_blocks=elastic_blocks,
                                         flags=(B.EKV_START_GROWN if start_grown else 0) | (B.EKV_FUSED_RANGE if fused_range else 0) |
-                                        (B.EKV_PREFILL_WARP_MMA if prefill_warp_mma else 0))
+                                        (B.EKV_PREFILL_WARP_MMA if prefill_warp_mma else 0) |
+                                        (B.EKV_PREFILL_ONE_HEAD if prefill_one_head else 0) |
+                                        (B.EKV_PREFILL_TWO_HEAD if prefill_two_head else 0))
         self.num_q_heads, self.num_kv_heads, self.head_dim, self.block_size = num_q_heads, num_kv_heads, head_dim, block_size
         self.num_layers = num_layers
         self._ws = None

@@ -39,9 +39,26 @@ def rand_q(seed, rows, shape):
         rows, shape.num_q_heads, shape.head_dim)
 
 
+# Which prefill kernel the pools of a test ask for (see the `prefill_kernel` fixture): nothing = the library's own
+# choice by shape and chunk length; otherwise one of the pool flags that pin it.
+_PREFILL_FLAGS = {}
+
+
 def make_pool(shape, base_blocks, elastic_blocks=0, grown=False, layers=1):
     return ekv.Pool(num_q_heads=shape.num_q_heads, num_kv_heads=shape.num_kv_heads, head_dim=shape.head_dim,
-                    base_blocks=base_blocks, elastic_blocks=elastic_blocks, num_layers=layers, start_grown=grown)
+                    base_blocks=base_blocks, elastic_blocks=elastic_blocks, num_layers=layers, start_grown=grown,
+                    **_PREFILL_FLAGS)
+
+
+@pytest.fixture(params=["auto", "one_head", "two_head", "warp_mma"])
+def prefill_kernel(request):
+    """Runs a prefill test once per kernel family: the library's own choice, then each family pinned through its pool
+    flag (two_head falls back to one_head on shapes it cannot take: head_dim 64, odd query groups)."""
+    _PREFILL_FLAGS.clear()
+    if request.param != "auto":
+        _PREFILL_FLAGS["prefill_" + request.param] = True
+    yield request.param
+    _PREFILL_FLAGS.clear()
 
 
 class Case:
@@ -316,7 +333,7 @@ def run_prefill(case, q, chunks, scale):
     return outs
 
 
-def test_prefill_c1_chunk_over_cached_prefix():
+def test_prefill_c1_chunk_over_cached_prefix(prefill_kernel):
     """configs[0]: one 256-token chunk over a 256-token cached prefix."""
     cfg = I.C1
     case = Case(cfg.shape, [512], 512, cfg.seed + 100, elastic_blocks=256)
@@ -334,8 +351,8 @@ def test_prefill_c1_chunk_over_cached_prefix():
         case.close()
 
 
-@pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY, I.LLAMA70B])
-def test_prefill_batched_ragged_requests_match_oracle(shape):
+@pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY, I.LLAMA70B, I.Shape(12, 4, 128), I.Shape(6, 2, 64)])
+def test_prefill_batched_ragged_requests_match_oracle(shape, prefill_kernel):
     chunks = [(0, 1), (0, 100), (37, 64), (500, 129), (130, 300), (1000, 17)]  # (prefix, rows)
     lengths = [p + c for p, c in chunks]
     need = int(I.blocks_for(torch.tensor(lengths), 16).sum())
@@ -357,7 +374,7 @@ def test_prefill_batched_ragged_requests_match_oracle(shape):
 
 
 @pytest.mark.parametrize("shape,R", [(I.LLAMA8B, 60), (I.TINY, 60), (I.LLAMA8B, 300)])
-def test_prefill_many_requests_find_their_tiles(shape, R):
+def test_prefill_many_requests_find_their_tiles(shape, R, prefill_kernel):
     """Many short requests in one call, some of them empty: every query tile must find its request (up to 256
     requests by bisection over a prefix table in the kernel parameters, more by walking cu_q_lens)."""
     rows = I.uniform_ints(71, 1, R, 0, 150)                  # chunk lengths, zeros included
@@ -381,7 +398,7 @@ def test_prefill_many_requests_find_their_tiles(shape, R):
 
 @pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY])
 @pytest.mark.parametrize("mult", [4, 16])
-def test_sharp_softmax_large_scores(shape, mult):
+def test_sharp_softmax_large_scores(shape, mult, prefill_kernel):
     """Queries 4x and 16x larger than the configs draw them: scores spread over tens of units, a row's running
     maximum jumps far between key tiles (the rescale paths of both kernels run), and nearly all the weight sits on a
     few keys.  Still inside the tolerance."""
@@ -403,7 +420,7 @@ def test_sharp_softmax_large_scores(shape, mult):
 
 
 @pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY])
-def test_scores_that_rise_along_the_sequence_force_a_rescale_at_every_tile(shape):
+def test_scores_that_rise_along_the_sequence_force_a_rescale_at_every_tile(shape, prefill_kernel):
     """Keys grow along the sequence so that each 16-token block scores about 2 units (log2) above the one before: a
     row's running maximum rises by far more than the lazy-rescale threshold at every key tile, the accumulated output
     is scaled down by 2^-16 or less each time, and nearly all the weight sits on the last visible block."""
@@ -431,7 +448,7 @@ def test_scores_that_rise_along_the_sequence_force_a_rescale_at_every_tile(shape
         case.close()
 
 
-def test_prefill_chunked_equals_one_shot_and_decode_equals_last_row():
+def test_prefill_chunked_equals_one_shot_and_decode_equals_last_row(prefill_kernel):
     shape = I.LLAMA8B
     L = 1500
     case = Case(shape, [L], 120, 71)
@@ -512,9 +529,9 @@ def test_elastic_toggle_bytes_pointer_and_outputs():
         pool.close()
 
 
-def test_prefill_edge_cases_bad_ids_empty_requests_and_both_kernels_agree():
-    """Out-of-range block ids inside a prompt are skipped and latched (both prefill kernels); requests with zero
-    rows are legal; the tcgen05 kernel and the warp-MMA kernel agree within tolerance on the same call."""
+def test_prefill_edge_cases_bad_ids_empty_requests_negative_scale(prefill_kernel):
+    """Out-of-range block ids inside a prompt are skipped and latched (every prefill kernel); requests with zero
+    rows are legal; a negative scale is served (by the warp-level kernel) whatever the pool asks for."""
     shape = I.LLAMA8B
     pool = make_pool(shape, 128, 32, grown=False)
     try:
@@ -554,12 +571,16 @@ def test_prefill_edge_cases_bad_ids_empty_requests_and_both_kernels_agree():
         assert pool.poll_status() == ekv.Status.OK
     finally:
         pool.close()
-    # the same call through each kernel family (a pool created with EKV_PREFILL_WARP_MMA always takes the warp-level
-    # kernel), each against the oracle and against the other
+
+
+def test_prefill_kernel_families_agree_on_the_same_call():
+    """The same call through each kernel family (pinned by its pool flag), each against the oracle and against the
+    others."""
+    shape = I.LLAMA8B
     outs = {}
-    for impl in ("mma", "tc"):
+    for impl in ("warp_mma", "two_head", "one_head"):
         pool = ekv.Pool(num_q_heads=shape.num_q_heads, num_kv_heads=shape.num_kv_heads, head_dim=shape.head_dim,
-                        base_blocks=64, prefill_warp_mma=(impl == "mma"))
+                        base_blocks=64, **{"prefill_" + impl: True})
         try:
             case = Case(shape, [700, 45], 64, 93, pool=pool)
             cu = torch.tensor([0, 300, 345], dtype=torch.int32)
@@ -571,9 +592,10 @@ def test_prefill_edge_cases_bad_ids_empty_requests_and_both_kernels_agree():
             assert pool.poll_status() == ekv.Status.OK
         finally:
             pool.close()
-    diff = (outs["mma"] - outs["tc"]).abs()
-    assert diff.max().item() <= MAX_ABS and diff.mean().item() <= MEAN_ABS
-    assert not torch.equal(outs["mma"], outs["tc"]), "two different kernels are expected to round differently somewhere"
+    for a, b in (("warp_mma", "two_head"), ("warp_mma", "one_head"), ("two_head", "one_head")):
+        diff = (outs[a] - outs[b]).abs()
+        assert diff.max().item() <= MAX_ABS and diff.mean().item() <= MEAN_ABS, (a, b)
+    assert not torch.equal(outs["warp_mma"], outs["two_head"]), "different kernels are expected to round differently somewhere"
 
 
 def test_recommit_out_of_memory_leaves_the_pool_shrunk_and_usable():

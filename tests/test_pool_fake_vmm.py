@@ -152,7 +152,7 @@ def test_failed_create_leaves_nothing_behind(vmm):
 
 def test_argument_checks_and_host_only_refusal(vmm):
     for bad in (dict(head_dim=96), dict(block_size=32), dict(num_q_heads=12, num_kv_heads=8),
-                dict(num_q_heads=72, num_kv_heads=8), dict(base_blocks=0), dict(elastic_blocks=-1), dict(flags=16)):
+                dict(num_q_heads=72, num_kv_heads=8), dict(base_blocks=0), dict(elastic_blocks=-1), dict(flags=64)):
         with pytest.raises(ekv.EkvError) as e:
             _create(**bad)
         assert e.value.status == ekv.Status.ERR_INVALID
