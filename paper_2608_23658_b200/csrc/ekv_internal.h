@@ -67,4 +67,9 @@ ekv_status_t launch_set_live(ekv_pool *pool, long long value, cudaStream_t strea
 ekv_status_t encode_kv_map(void *base, uint64_t blocks, uint64_t block_stride, int num_kv_heads, int head_dim, int block_size,
                            CUtensorMap *out);
 
+// Tensor map over a query tensor [tokens, num_q_heads, head_dim] bf16: dims (channel, head, token), box 64 channels x
+// 1 head x box_rows tokens, 128-byte swizzle: one box lands as the K-major [row][128 B] half tile the MMAs read.
+// Tokens past the end read as zero.
+ekv_status_t encode_q_map(const void *q, uint64_t tokens, int num_q_heads, int head_dim, int box_rows, CUtensorMap *out);
+
 }  // namespace ekv

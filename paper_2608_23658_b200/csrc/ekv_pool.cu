@@ -194,6 +194,23 @@ ekv_status_t encode_kv_map(void *base, uint64_t blocks, uint64_t block_stride, i
     return EKV_OK;
 }
 
+ekv_status_t encode_q_map(const void *q, uint64_t tokens, int num_q_heads, int head_dim, int box_rows, CUtensorMap *out) {
+    if (!load_driver()) return EKV_ERR_CUDA;
+    cuuint64_t gdim[3] = {(cuuint64_t)head_dim, (cuuint64_t)num_q_heads, (cuuint64_t)tokens};
+    cuuint64_t gstride[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)num_q_heads * head_dim * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_drv.encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(q), gdim, gstride, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled failed (CUresult %d) for a query tensor at %p with %llu tokens", (int)r, q,
+                  (unsigned long long)tokens);
+        return EKV_ERR_CUDA;
+    }
+    return EKV_OK;
+}
+
 static uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
 
 static double now_ms() {

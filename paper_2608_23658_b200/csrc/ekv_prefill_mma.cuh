@@ -25,6 +25,7 @@ struct PrefillParams {
     unsigned *status;
     int *abort_word;  // device word: a CTA of this launch gave up on a wait (tcgen05 kernel)
     int max_blocks, num_q_heads, num_kv_heads, group, R;
+    int q_tiles;      // query tiles of the call (of the launching kernel's tile height)
     float scale_log2;
     // tile_prefix[r] = query tiles of requests 0..r-1 (filled by the host when R <= kPrefixMax, else n_prefix = 0):
     // lets a CTA find its request by bisection in the parameter bank instead of walking cu_q_lens

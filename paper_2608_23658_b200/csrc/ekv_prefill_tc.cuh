@@ -1,22 +1,36 @@
 // Chunked-prefill attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM),
-// head_dim 128, even query group.
+// head_dim 128, even query group.  PERSISTENT: one CTA per SM walks a list of work items.
 //
-// One CTA = 128 query positions of one request x TWO query heads (A, B) that share a kv-head, so
+// Work item = 128 query positions of one request x TWO query heads (A, B) that share a kv-head, so
 // every K/V tile staged in shared memory feeds two 128x128 score tiles (ping-pong: while the
-// softmax warps work on one head's scores the tensor pipe runs the other head's MMAs).
+// softmax warps work on one head's scores the tensor pipe runs the other head's MMAs).  Items are
+// ordered head pair by head pair and, inside a pair, from the heaviest (latest) query tile to the
+// lightest, and are handed out dynamically: warp 3 draws item numbers from a counter in device
+// memory and posts them in a small ring in shared memory, from which every role of the CTA reads
+// its next item (longest-first greedy scheduling; a static round-robin would give CTA c the same
+// position of every request whenever the request length divides the grid).  All roles walk that
+// list independently and are only coupled through mbarriers, so the end of one item overlaps the
+// start of the next:
+// the Q tiles and first K/V tiles of item i+1 are in flight during the last tiles of item i, the
+// first QK^T of item i+1 is issued right behind the last PV of item i, and the write-out of item i
+// runs while the tensor pipe already works on item i+1.  TMEM and the barriers are set up once.
 //
-//   warp 0        TMA producer: 16-token x 64-channel boxes (128-byte swizzle) of K and V blocks,
-//                 gathered through the block table into 128-key tiles, 2 stages each for K and V
-//   warp 1        MMA issuer (whole warp converged, one elected lane issues): S = Q K^T (A, B from shared memory, K-major) and
-//                 O += P V (A = P read from TMEM, B = V from shared memory, MN-major)
-//   warp 2        TMEM allocation / release (512 columns: S_A S_B O_A O_B, P aliases S)
-//   warps 4-7     softmax of head A: one thread per query row (= TMEM lane)
-//   warps 8-11    softmax of head B
+//   warp 0        TMA producer of K tiles: 16-token x 64-channel boxes (128-byte swizzle) of the
+//                 blocks the table names, gathered into 128-key tiles, 2 stages
+//   warp 1        MMA issuer (whole warp converged, one elected lane issues): S = Q K^T (A, B from
+//                 shared memory, K-major) and O += P V (A = P read from TMEM, B = V from shared
+//                 memory, MN-major)
+//   warp 2        TMA producer of V tiles, 2 stages; TMEM allocation / release (512 columns:
+//                 S_A S_B O_A O_B, P aliases S)
+//   warp 3        item scheduler; TMA producer of the two Q tiles of an item (one tensor map over
+//                 the query tensor)
+//   warps 4-7     softmax of head A: one thread per query row (= TMEM lane); write-out of head A
+//   warps 8-11    softmax and write-out of head B
 //
 // Softmax is online in the exp2 domain with LAZY rescaling: the running reference max of a row is
 // only raised (and O, l rescaled in TMEM) when a tile's max exceeds it by more than 2^8, so P stays
 // below 256 and most tiles need no pass over O.  All mbarrier waits are bounded; a wait that runs
-// out latches EKV_ERR_TIMEOUT, makes every role leave its loop, and the CTA still drains its
+// out latches EKV_ERR_TIMEOUT, makes every role leave its loops, and the CTA still drains its
 // copies, releases TMEM and exits.
 #pragma once
 #include <cuda/ptx>
@@ -26,6 +40,13 @@
 #include "ekv_internal.h"
 #include "ekv_prefill_mma.cuh"  // PrefillParams
 #include "ptx.cuh"
+
+#ifndef EKV_TC_PAIR_GROUP
+#define EKV_TC_PAIR_GROUP 0
+#endif
+#ifndef EKV_TC_ITEM_AHEAD
+#define EKV_TC_ITEM_AHEAD 1
+#endif
 
 namespace ekv {
 namespace tc {
@@ -42,7 +63,8 @@ static constexpr int kThreads = 384;
 static constexpr float kRescaleThreshold = 8.f;        // log2 units
 // Register re-partition (setmaxnreg): the CTA owns kLaunchRegs x kThreads registers.  Warps 0-3 drop to
 // kRegsUtil, warps 4-11 rise to kRegsSoftmax.  The raise BLOCKS until the pool has the registers, so
-// the split must fit the CTA's own allocation exactly -- nothing else bounds that wait.
+// the split must fit the CTA's own allocation exactly -- nothing else bounds that wait -- and every
+// warpgroup (four consecutive warps from a multiple of four) must ask for the same thing.
 static constexpr int kLaunchRegs = 168, kRegsUtil = 72, kRegsSoftmax = 216;
 static_assert(128 * kRegsUtil + 256 * kRegsSoftmax <= kLaunchRegs * kThreads, "setmaxnreg split exceeds the CTA's registers");
 static_assert(kLaunchRegs * kThreads <= 65536 && kRegsUtil % 8 == 0 && kRegsSoftmax % 8 == 0, "register split");
@@ -51,11 +73,18 @@ static_assert(kLaunchRegs * kThreads <= 65536 && kRegsUtil % 8 == 0 && kRegsSoft
 static constexpr int kOffQ = 0;                                   // Q_A, Q_B
 static constexpr int kOffK = kOffQ + 2 * kTileBytes;              // K stages
 static constexpr int kOffV = kOffK + kStages * kTileBytes;        // V stages
-static constexpr int kOffBar = kOffV + kStages * kTileBytes;      // mbarriers
+static constexpr int kOffStage = kOffV + kStages * kTileBytes;    // write-out staging: 8 softmax warps x [32 rows][128 B]
+static constexpr int kStageBytes = 32 * 128;
+static constexpr int kOffBar = kOffStage + 8 * kStageBytes;       // mbarriers
 static constexpr int kSmemBytes = kOffBar + 256 + 1024;           // + alignment slack
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
 // barrier slots (8 bytes each)
-enum Bar { Q_READY = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_READY = 9, P_READY = 11, DRAIN = 13, P_PART = 14, NBAR = 16 };
+static constexpr int kItemRing = 4;   // item numbers posted ahead of the slowest role
+static constexpr int kItemAhead = EKV_TC_ITEM_AHEAD;  // the scheduler keeps this many items posted beyond the one whose Q it loads
+enum Bar { Q_FULL = 0, Q_EMPTY = 2, K_FULL = 4, K_EMPTY = 6, V_FULL = 8, V_EMPTY = 10, S_READY = 12, P_READY = 14, P_PART = 16,
+           O_FREE = 18, DRAIN = 20, ITEM_READY = 21, ITEM_DONE = ITEM_READY + kItemRing, NBAR = ITEM_DONE + 1 };
+static_assert(8 * NBAR + 32 + 4 * kItemRing <= 256, "barrier area");
 
 // TMEM columns
 __device__ __forceinline__ constexpr uint32_t col_s(int x) { return 128u * (uint32_t)x; }
@@ -125,10 +154,12 @@ struct Shared {
     __device__ __forceinline__ uint32_t bar(int i) const { return base + kOffBar + 8 * i; }
     __device__ __forceinline__ volatile int *abort_flag() const { return (volatile int *)(ptr + kOffBar + 8 * NBAR); }
     __device__ __forceinline__ uint32_t *tmem_slot() const { return (uint32_t *)(ptr + kOffBar + 8 * NBAR + 8); }
-    // Per-tile mask of key blocks whose shared-memory rows hold stand-in data.  Ring of 4: the K producer
-    // may run two tiles ahead of the softmax warps (it only waits for the QK MMAs), so a slot per STAGE
-    // would be overwritten before the softmax of the older tile has read it.
+    // Per-tile mask of key blocks whose shared-memory rows hold stand-in data.  Ring of 4, indexed by the CTA's running
+    // key-tile count: the K producer may run two tiles ahead of the softmax warps (it only waits for the QK MMAs), so a
+    // slot per STAGE would be overwritten before the softmax of the older tile has read it.
     __device__ __forceinline__ volatile int *bad_mask(int tile) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 16 + 4 * (tile & 3)); }
+    // item numbers posted by the scheduler: slot k % kItemRing holds the CTA's k-th item
+    __device__ __forceinline__ volatile int *item_slot(int k) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 32 + 4 * (k % kItemRing)); }
 };
 
 // Bounded wait that also gives up as soon as another role has flagged an abort.
@@ -156,37 +187,56 @@ __device__ __forceinline__ bool wait_warp(const Shared &sh, int bar, uint32_t pa
     return __all_sync(0xffffffffu, wait_or_abort(sh, bar, parity, status, abort_word));
 }
 
-__global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_constant__ CUtensorMap kvmap,
-                                                                 const PrefillParams p) {
-    // a CTA of an earlier wave of this launch already timed out: do not start more work (the flag lives
-    // in device memory and is cleared by the launcher; the host-mapped status word is never polled here)
-    if (*(volatile int *)p.abort_word) return;
+// The CTA's k-th item number, as posted by the scheduler (a number >= the item count ends the list); -1 if the wait
+// was given up.
+__device__ __forceinline__ int fetch_item(const Shared &sh, int k, unsigned *status, int *abort_word) {
+    if (!wait_warp(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1), status, abort_word)) return -1;
+    return *sh.item_slot(k);
+}
 
-    // ---- which (request, 128-row tile, head pair)?  Heaviest (latest) tiles first.
-    const int tile_idx = gridDim.x - 1 - blockIdx.x;
-    const int pair = blockIdx.y;
-    const int head0 = 2 * pair;
-    const int g = head0 / p.group;
-    int req = 0, acc_tiles = 0, c_r = 0, q0 = 0;
-    if (!find_request(p, tile_idx, kBM, req, acc_tiles, q0, c_r)) return;
-    const int row0 = (tile_idx - acc_tiles) * kBM;
-    const int L = min(p.seq_lens[req], p.max_blocks * 16);
-    const int prefix = L - c_r;
-    const int rows_here = min(kBM, c_r - row0);
+// One work item, decoded the same way by every role.
+struct Item {
+    int req, q0, row0, rows_here, L, prefix, n_tiles, n_blocks, head0, g;
+    bool malformed;  // seq_len shorter than the chunk: rows are zero-filled, nothing is loaded or multiplied
+};
+// Item order: head pairs are taken in groups of kPairGroup (0 = all pairs in one group); inside a group the query tiles
+// go from the heaviest (latest) to the lightest and every tile is listed for all pairs of the group before the next
+// tile.  One group per launch makes the list globally longest-first (the end of the launch is made of one-tile items,
+// so the CTAs finish together); smaller groups keep fewer kv-heads' K/V streaming through L2 at a time.
+static constexpr int kPairGroup = EKV_TC_PAIR_GROUP;
+__device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item &it) {
+    const int npairs = p.num_q_heads / 2;
+    const int gp = kPairGroup > 0 ? kPairGroup : npairs;
+    const int per_group = p.q_tiles * gp;
+    const int grp = m / per_group, r = m - grp * per_group;
+    const int in_group = min(gp, npairs - grp * gp);       // the last group may be smaller
+    const int rank = r / in_group;
+    const int pair = grp * gp + (r - rank * in_group);
+    const int tile_idx = p.q_tiles - 1 - rank;              // heaviest (latest) tiles first
+    int acc_tiles = 0, c_r = 0;
+    if (!find_request(p, tile_idx, kBM, it.req, acc_tiles, it.q0, c_r)) return false;
+    it.head0 = 2 * pair;
+    it.g = it.head0 / p.group;
+    it.row0 = (tile_idx - acc_tiles) * kBM;
+    it.L = min(p.seq_lens[it.req], p.max_blocks * 16);
+    it.prefix = it.L - c_r;
+    it.rows_here = min(kBM, c_r - it.row0);
+    it.malformed = it.prefix < 0;
+    const int kv_end = min(it.L, it.prefix + it.row0 + it.rows_here);  // keys any row of this tile may see
+    it.n_tiles = (kv_end + kBN - 1) / kBN;
+    it.n_blocks = (kv_end + 15) >> 4;
+    return true;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_constant__ CUtensorMap kvmap,
+                                                                 const __grid_constant__ CUtensorMap qmap,
+                                                                 const PrefillParams p) {
+    // a CTA of this launch already timed out: do not start more work (the flag lives in device memory and is
+    // cleared by the launcher; the host-mapped status word is never polled here)
+    if (*(volatile int *)p.abort_word) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t row_stride = (size_t)p.num_q_heads * kD;
-
-    if (prefix < 0) {  // malformed request: zero rows, latch
-        if (threadIdx.x == 0) atomicOr(p.status, EKV_DEV_FLAG_OOB);
-        for (int e = threadIdx.x; e < rows_here * 2 * kD; e += kThreads) {
-            const int row = e / (2 * kD), x = e % (2 * kD);
-            p.out[((size_t)(q0 + row0 + row)) * row_stride + (size_t)head0 * kD + x] = __float2bfloat16_rn(0.f);
-        }
-        return;
-    }
-    const int kv_end = min(L, prefix + row0 + rows_here);  // keys any row of this tile may see
-    const int n_tiles = (kv_end + kBN - 1) / kBN;
-    const int n_blocks = (kv_end + 15) >> 4;
+    const int n_items = p.q_tiles * (p.num_q_heads / 2);
 
     extern __shared__ uint8_t smem_raw[];
     Shared sh;
@@ -198,19 +248,24 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
 
     if (threadIdx.x == 0) {
         prefetch_tensormap(&kvmap);
-        mbar_init(sh.bar(Q_READY), 256);
+        prefetch_tensormap(&qmap);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(sh.bar(Q_FULL + x), 1);
+            mbar_init(sh.bar(Q_EMPTY + x), 1);
+            mbar_init(sh.bar(S_READY + x), 1);
+            mbar_init(sh.bar(P_READY + x), 128);
+            mbar_init(sh.bar(P_PART + x), 128);
+            mbar_init(sh.bar(O_FREE + x), 4);
+        }
         for (int s = 0; s < kStages; ++s) {
             mbar_init(sh.bar(K_FULL + s), 1);
             mbar_init(sh.bar(K_EMPTY + s), 1);
             mbar_init(sh.bar(V_FULL + s), 1);
             mbar_init(sh.bar(V_EMPTY + s), 1);
         }
-        for (int x = 0; x < 2; ++x) {
-            mbar_init(sh.bar(S_READY + x), 1);
-            mbar_init(sh.bar(P_READY + x), 128);
-            mbar_init(sh.bar(P_PART + x), 128);
-        }
         mbar_init(sh.bar(DRAIN), 1);
+        for (int i = 0; i < kItemRing; ++i) mbar_init(sh.bar(ITEM_READY + i), 1);
+        mbar_init(sh.bar(ITEM_DONE), 8);
         *sh.abort_flag() = 0;
         mbar_fence_init();
     }
@@ -222,6 +277,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     __syncthreads();
     fence_after();
     const uint32_t tmem = *sh.tmem_slot();
+    // what this warp has put in flight (producers only): the teardown of an aborted CTA waits for the last of it
+    int tiles_issued = 0;
 
     if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
@@ -233,42 +290,103 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         const uint32_t tile_base = sh.base + (is_v ? kOffV : kOffK);
         const int kv_row_off = is_v ? p.num_kv_heads * 16 : 0;
         const long long live = *p.live;
-        const int *bt = p.block_tables + (size_t)req * p.max_blocks;
-        auto load_id = [&](int j) {  // lane l: id of block 8j + l%8 (-1 past the end, -2 invalid)
-            int id = -1;
-            const int bi = 8 * j + (lane & 7);
-            if (bi < n_blocks) {
-                id = bt[bi];
-                if (id < 0 || (long long)id >= live) id = -2;
-            }
-            return id;
-        };
-        int id_next = load_id(0);
-        for (int j = 0; j < n_tiles; ++j) {
-            const int s = j % kStages;
-            const int id_raw = id_next;
-            if (j + 1 < n_tiles) id_next = load_id(j + 1);
-            const unsigned oob = __ballot_sync(0xffffffffu, id_raw == -2) & 0xffu;
-            // blocks whose smem rows will hold stand-in data: invalid ids and blocks past the last visible key
-            const unsigned bad = __ballot_sync(0xffffffffu, id_raw < 0) & 0xffu;
-            const int id = id_raw < 0 ? 0 : id_raw;  // masked later; block 0 is always mapped
-            // box b of a tile: block b/2, channel half b%2  ->  [half][block][16 rows][128 B]
-            const int b = lane & 15, blk = b >> 1, half = b & 1;
-            const int my_id = __shfl_sync(0xffffffffu, id, blk);
-            const int row = g * 16 + kv_row_off;  // row inside the block: (K|V, kv-head, token)
-            if (j >= kStages && !wait_warp(sh, EMPTY + s, (uint32_t)(((j / kStages) - 1) & 1), p.status, p.abort_word)) break;
-            if (lane == 0) {
-                if (!is_v) {
-                    if (oob) atomicOr(p.status, EKV_DEV_FLAG_OOB);
-                    *sh.bad_mask(j) = (int)bad;
+        int t = 0;  // tiles issued so far (all items): stage t % kStages, use number t / kStages of that stage
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+            const int m = fetch_item(sh, k, p.status, p.abort_word);
+            if (m < 0 || m >= n_items) break;
+            Item it;
+            if (!decode_item(p, m, it) || it.malformed) continue;
+            const int *bt = p.block_tables + (size_t)it.req * p.max_blocks;
+            auto load_id = [&](int j) {  // lane l: id of block 8j + l%8 (-1 past the end, -2 invalid)
+                int id = -1;
+                const int bi = 8 * j + (lane & 7);
+                if (bi < it.n_blocks) {
+                    id = bt[bi];
+                    if (id < 0 || (long long)id >= live) id = -2;
                 }
-                mbar_expect_tx(sh.bar(FULL + s), kTileBytes);
+                return id;
+            };
+            int id_next = load_id(0);
+            for (int j = 0; j < it.n_tiles; ++j, ++t) {
+                const int s = t % kStages;
+                const int id_raw = id_next;
+                if (j + 1 < it.n_tiles) id_next = load_id(j + 1);
+                const unsigned oob = __ballot_sync(0xffffffffu, id_raw == -2) & 0xffu;
+                // blocks whose smem rows will hold stand-in data: invalid ids and blocks past the last visible key
+                const unsigned bad = __ballot_sync(0xffffffffu, id_raw < 0) & 0xffu;
+                const int id = id_raw < 0 ? 0 : id_raw;  // masked later; block 0 is always mapped
+                // box b of a tile: block b/2, channel half b%2  ->  [half][block][16 rows][128 B]
+                const int b = lane & 15, blk = b >> 1, half = b & 1;
+                const int my_id = __shfl_sync(0xffffffffu, id, blk);
+                const int row = it.g * 16 + kv_row_off;  // row inside the block: (K|V, kv-head, token)
+                if (t >= kStages && !wait_warp(sh, EMPTY + s, (uint32_t)(((t / kStages) - 1) & 1), p.status, p.abort_word)) {
+                    ok = false;
+                    break;
+                }
+                if (lane == 0) {
+                    if (!is_v) {
+                        if (oob) atomicOr(p.status, EKV_DEV_FLAG_OOB);
+                        *sh.bad_mask(t) = (int)bad;
+                    }
+                    mbar_expect_tx(sh.bar(FULL + s), kTileBytes);
+                }
+                __syncwarp();
+                if (lane < 16)
+                    tma_load_3d(tile_base + s * kTileBytes + half * kHalfBytes + blk * 2048, &kvmap, 64 * half, row, my_id, sh.bar(FULL + s));
             }
-            __syncwarp();
-            if (lane < 16)
-                tma_load_3d(tile_base + s * kTileBytes + half * kHalfBytes + blk * 2048, &kvmap, 64 * half, row, my_id, sh.bar(FULL + s));
         }
-    } else if (warp == 1) {
+        tiles_issued = t;
+    } else if (warp == 3) {
+        // =========================== item scheduler + TMA producer of the Q tiles ===========================
+        int n = 0;       // well-formed items whose Q tiles were requested so far
+        int posted = 0;  // item numbers posted so far
+        bool ok = true, drained = false;
+        int *counter = p.abort_word + 1;  // next item number of the launch (cleared by the launcher with the abort word)
+        // Post item numbers up to the CTA's `upto`-th.  Slot k % kItemRing is free again once the CTA's item
+        // k - kItemRing is written out: every role has long read it by then.
+        auto post_until = [&](int upto) -> bool {
+            while (posted <= upto && !drained) {
+                if (posted >= kItemRing &&
+                    !wait_warp(sh, ITEM_DONE, (uint32_t)((posted - kItemRing) & 1), p.status, p.abort_word))
+                    return false;
+                int m = 0;
+                if (lane == 0) {
+                    m = atomicAdd(counter, 1);
+                    *sh.item_slot(posted) = m;
+                    __threadfence_block();
+                    mbar_arrive(sh.bar(ITEM_READY + posted % kItemRing));
+                }
+                m = __shfl_sync(0xffffffffu, m, 0);
+                drained = m >= n_items;  // the end marker is posted once; nobody reads past it
+                ++posted;
+            }
+            return true;
+        };
+        for (int k = 0; ok; ++k) {
+            ok = post_until(k + kItemAhead);
+            if (!ok) break;
+            const int m = *sh.item_slot(k);  // posted by this warp (k < posted always holds here unless the list ended before k)
+            if (k >= posted || m >= n_items) break;
+            Item it;
+            if (!decode_item(p, m, it) || it.malformed) continue;
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                // the previous item's last QK^T of this head has read the tile
+                if (n > 0 && !wait_warp(sh, Q_EMPTY + x, (uint32_t)((n - 1) & 1), p.status, p.abort_word)) {
+                    ok = false;
+                    break;
+                }
+                if (lane == 0) mbar_expect_tx(sh.bar(Q_FULL + x), kTileBytes);
+                __syncwarp();
+                if (lane < 2)  // rows past the end of the query tensor read as zero; rows past the request's chunk are never written out
+                    tma_load_3d(sh.base + kOffQ + x * kTileBytes + lane * kHalfBytes, &qmap, 64 * lane, it.head0 + x, it.q0 + it.row0,
+                                sh.bar(Q_FULL + x));
+            }
+            if (ok) ++n;
+        }
+        tiles_issued = n;
+    } else {
         // =========================== MMA issuer ===========================
         // descriptor low words of the tile origins; stepping inside a tile adds a compile-time constant
         const uint32_t q_lo[2] = {desc_lo(sh.base + kOffQ, 16), desc_lo(sh.base + kOffQ + kTileBytes, 16)};
@@ -288,44 +406,85 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             for (int k = k0; k < k1; ++k)
                 mma_ts_lo_dyn(tmem + col_o(x), tmem + col_s(x) + 8 * k, v_lo + ((k * 2048) >> 4), kIdescPV, (acc || k > 0) ? 1u : 0u);
         };
-        bool ok = wait_warp(sh, Q_READY, 0, p.status, p.abort_word) && wait_warp(sh, K_FULL + 0, 0, p.status, p.abort_word);
-        if (ok) {
-            fence_after();
-            issue_qk(0, 0);
-            mma_commit(sh.bar(S_READY + 0));
-            issue_qk(1, 0);
-            mma_commit(sh.bar(K_EMPTY + 0));
-            mma_commit(sh.bar(S_READY + 1));
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int s = j % kStages, s1 = (j + 1) % kStages;
-                const bool more = j + 1 < n_tiles;
-                ok = wait_warp(sh, V_FULL + s, (uint32_t)((j / kStages) & 1), p.status, p.abort_word);
-                if (ok && more) ok = wait_warp(sh, K_FULL + s1, (uint32_t)(((j + 1) / kStages) & 1), p.status, p.abort_word);
-                if (ok) ok = wait_warp(sh, P_PART + 0, (uint32_t)(j & 1), p.status, p.abort_word);
-                if (!ok) break;
-                fence_after();
-                issue_pv(0, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
-                ok = wait_warp(sh, P_READY + 0, (uint32_t)(j & 1), p.status, p.abort_word);
-                if (!ok) break;
-                fence_after();
-                issue_pv(0, s, true, kPartSteps, kBN / 16);
-                if (more) issue_qk(0, s1);
-                mma_commit(sh.bar(S_READY + 0));
-                ok = wait_warp(sh, P_PART + 1, (uint32_t)(j & 1), p.status, p.abort_word);
-                if (!ok) break;
-                fence_after();
-                issue_pv(1, s, j > 0, 0, kPartSteps);
-                ok = wait_warp(sh, P_READY + 1, (uint32_t)(j & 1), p.status, p.abort_word);
-                if (!ok) break;
-                fence_after();
-                issue_pv(1, s, true, kPartSteps, kBN / 16);
-                mma_commit(sh.bar(V_EMPTY + s));
-                if (more) {
-                    issue_qk(1, s1);
-                    mma_commit(sh.bar(K_EMPTY + s1));
-                }
-                mma_commit(sh.bar(S_READY + 1));
+        // The item list of this CTA, one item ahead: the first QK^T of the next item is issued inside the last
+        // key tile of the current one.
+        int k_item = 0;
+        bool list_ok = true, list_end = false;
+        Item cur, nxt;
+        bool have_cur = false, have_nxt = false;
+        auto advance = [&](Item &it, bool &have) {  // next well-formed item of this CTA, if any
+            have = false;
+            while (list_ok && !list_end && !have) {
+                const int m = fetch_item(sh, k_item++, p.status, p.abort_word);
+                if (m < 0) list_ok = false;
+                else if (m >= n_items) list_end = true;
+                else have = decode_item(p, m, it) && !it.malformed;
             }
+        };
+        advance(cur, have_cur);
+        int t = 0;   // key tiles whose QK^T (both heads) has been issued: the next QK^T reads K stage t % kStages
+        int tv = 0;  // key tiles whose PV has been issued
+        int n = 0;   // items whose first QK^T has been issued
+        bool ok = have_cur && list_ok;
+        // first QK^T of an item: its Q tile of head x and (checked for head A) the K tile must have landed
+        auto first_qk = [&](int x, const Item &it) -> bool {
+            if (!wait_warp(sh, Q_FULL + x, (uint32_t)(n & 1), p.status, p.abort_word)) return false;
+            if (x == 0 && !wait_warp(sh, K_FULL + t % kStages, (uint32_t)((t / kStages) & 1), p.status, p.abort_word)) return false;
+            fence_after();
+            issue_qk(x, t % kStages);
+            if (it.n_tiles == 1) mma_commit(sh.bar(Q_EMPTY + x));  // also the item's last QK^T of this head
+            return true;
+        };
+        if (ok) {
+            ok = first_qk(0, cur);
+            if (ok) mma_commit(sh.bar(S_READY + 0));
+            if (ok) ok = first_qk(1, cur);
+            if (ok) {
+                mma_commit(sh.bar(K_EMPTY + t % kStages));
+                mma_commit(sh.bar(S_READY + 1));
+                ++t;
+                ++n;
+            }
+        }
+        while (ok) {
+            advance(nxt, have_nxt);
+            if (!list_ok) break;
+            for (int j = 0; j < cur.n_tiles && ok; ++j, ++tv) {
+                const int s = tv % kStages;
+                const bool last = j + 1 == cur.n_tiles;
+                const bool more = !last || have_nxt;             // another key tile follows (this item's or the next one's)
+                const int s1 = t % kStages;                      // its stage
+                ok = wait_warp(sh, V_FULL + s, (uint32_t)((tv / kStages) & 1), p.status, p.abort_word);
+                if (ok && !last) ok = wait_warp(sh, K_FULL + s1, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    if (!ok) break;
+                    // O_x still holds the previous item's result until its write-out has read it
+                    if (j == 0 && n > 1) ok = wait_warp(sh, O_FREE + x, (uint32_t)((n - 2) & 1), p.status, p.abort_word);
+                    if (ok) ok = wait_warp(sh, P_PART + x, (uint32_t)(tv & 1), p.status, p.abort_word);
+                    if (!ok) break;
+                    fence_after();
+                    issue_pv(x, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
+                    ok = wait_warp(sh, P_READY + x, (uint32_t)(tv & 1), p.status, p.abort_word);
+                    if (!ok) break;
+                    fence_after();
+                    issue_pv(x, s, true, kPartSteps, kBN / 16);
+                    if (x == 1) mma_commit(sh.bar(V_EMPTY + s));
+                    if (!last) {
+                        issue_qk(x, s1);
+                        if (j + 2 == cur.n_tiles) mma_commit(sh.bar(Q_EMPTY + x));  // the item's last QK^T of this head
+                    } else if (have_nxt) {
+                        ok = first_qk(x, nxt);
+                        if (!ok) break;
+                    }
+                    if (x == 1 && more) mma_commit(sh.bar(K_EMPTY + s1));
+                    mma_commit(sh.bar(S_READY + x));  // scores of the next tile, and (after the last tile) O_x complete
+                }
+                if (ok && more) ++t;
+                if (ok && last && have_nxt) ++n;
+            }
+            if (!ok || !have_nxt) break;
+            cur = nxt;
         }
         // every MMA this thread issued must be finished before TMEM is released
         mma_commit(sh.bar(DRAIN));
@@ -333,173 +492,189 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-        // =========================== softmax + epilogue ===========================
+        // =========================== softmax + write-out ===========================
         const int x = (warp - 4) >> 2;                  // 0 = head A, 1 = head B
-        const int row = ((warp & 3) << 5) | lane;        // query row in the tile = TMEM lane
-        const int head = head0 + x;
-        const uint32_t lane_base = (uint32_t)((warp & 3) << 5) << 16;
+        const int wrow0 = (warp & 3) << 5;               // this warp's 32 rows of the tile = its TMEM lanes
+        const int row = wrow0 | lane;                    // query row in the tile = TMEM lane
+        const uint32_t lane_base = (uint32_t)wrow0 << 16;
         const uint32_t t_s = tmem + lane_base + col_s(x);
         const uint32_t t_o = tmem + lane_base + col_o(x);
+        uint8_t *stage = sh.ptr + kOffStage + (warp - 4) * kStageBytes;
 
-        // ---- stage this head's Q tile (128-byte swizzle).  Each warp brings in the 32 rows it will own, two rows per
-        // instruction: 16 lanes cover the 256 contiguous bytes of a row, so global loads are fully coalesced
-        // (one row per lane would touch 32 cache lines per instruction and cost microseconds per CTA).
-        const int wrow0 = (warp & 3) << 5;
-        {
-            uint8_t *qdst = sh.ptr + kOffQ + x * kTileBytes;
-            const int c16 = lane & 15;
-            const __nv_bfloat16 *src = p.q + ((size_t)(q0 + row0)) * row_stride + (size_t)head * kD + c16 * 8;
-            uint4 v[16];
-#pragma unroll
-            for (int it = 0; it < 16; ++it) {
-                const int rr = wrow0 + 2 * it + (lane >> 4);
-                v[it] = rr < rows_here ? *reinterpret_cast<const uint4 *>(src + (size_t)rr * row_stride) : make_uint4(0u, 0u, 0u, 0u);
+        // S_READY_x completes once per key tile of the CTA (all items), plus once after the very last PV: completion
+        // number t carries the scores of key tile t, and for the first tile of an item also "the previous item's O_x is
+        // complete" -- so the wait that ends an item is the wait that starts the next one.
+        int t = 0;  // key tiles processed so far (all items)
+        bool ok = true, waited = false;
+        auto item_done = [&]() {  // this warp is through with the item: its slot in the ring may be reused
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sh.bar(ITEM_DONE));
+        };
+        for (int k = 0; ok; ++k) {
+            const int m = fetch_item(sh, k, p.status, p.abort_word);
+            if (m < 0 || m >= n_items) break;
+            Item it;
+            if (!decode_item(p, m, it)) {
+                item_done();
+                continue;
             }
-#pragma unroll
-            for (int it = 0; it < 16; ++it) {
-                const int rr = wrow0 + 2 * it + (lane >> 4);
-                *reinterpret_cast<uint4 *>(qdst + (c16 >> 3) * kHalfBytes + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4)) = v[it];
+            const int head = it.head0 + x;
+            if (it.malformed) {  // zero rows, latch
+                if (threadIdx.x == 128) atomicOr(p.status, EKV_DEV_FLAG_OOB);
+                for (int e = threadIdx.x - 128 - 128 * x; e < it.rows_here * kD; e += 128)
+                    p.out[((size_t)(it.q0 + it.row0 + e / kD)) * row_stride + (size_t)head * kD + e % kD] = __float2bfloat16_rn(0.f);
+                item_done();
+                continue;
             }
-            fence_proxy_async_smem();
-            mbar_arrive(sh.bar(Q_READY));
-        }
-
-        const int lim = prefix + row0 + min(row, rows_here - 1);  // last key this row may see
-        float m_run = -INFINITY, l_run = 0.f;
-        bool ok = true;
-        for (int j = 0; j < n_tiles; ++j) {
-            const int s = j % kStages;
-            ok = wait_warp(sh, S_READY + x, (uint32_t)(j & 1), p.status, p.abort_word);
-            if (!ok) break;
-            fence_after();
-            const int key0 = j * kBN;
-            const int bad = *sh.bad_mask(j);
-            const bool need_mask = (key0 + kBN - 1 > prefix + row0) || bad != 0;
-            // keys of this tile that lie past the sequence end, or in a skipped block, may hold anything
-            // (unwritten slots): their V rows must not reach the tensor pipe, because 0 * NaN = NaN
-            const bool dirty_v = (key0 + kBN > L) || bad != 0;
-            if (dirty_v && x == 0) {
-                ok = wait_warp(sh, V_FULL + s, (uint32_t)((j / kStages) & 1), p.status, p.abort_word);
+            const int lim = it.prefix + it.row0 + min(row, it.rows_here - 1);  // last key this row may see
+            float m_run = -INFINITY, l_run = 0.f;
+            for (int j = 0; j < it.n_tiles; ++j, ++t) {
+                const int s = t % kStages;
+                if (!waited) ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
+                waited = false;
                 if (!ok) break;
-                uint8_t *vdst = sh.ptr + kOffV + s * kTileBytes;
-                if ((key0 + row >= L) || ((bad >> (row >> 4)) & 1)) {  // thread `row` owns key row `row` of the tile
+                fence_after();
+                const int key0 = j * kBN;
+                const int bad = *sh.bad_mask(t);
+                const bool need_mask = (key0 + kBN - 1 > it.prefix + it.row0) || bad != 0;
+                // keys of this tile that lie past the sequence end, or in a skipped block, may hold anything
+                // (unwritten slots): their V rows must not reach the tensor pipe, because 0 * NaN = NaN
+                const bool dirty_v = (key0 + kBN > it.L) || bad != 0;
+                if (dirty_v && x == 0) {
+                    ok = wait_warp(sh, V_FULL + s, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
+                    if (!ok) break;
+                    uint8_t *vdst = sh.ptr + kOffV + s * kTileBytes;
+                    if ((key0 + row >= it.L) || ((bad >> (row >> 4)) & 1)) {  // thread `row` owns key row `row` of the tile
 #pragma unroll
-                    for (int h2 = 0; h2 < 2; ++h2)
+                        for (int h2 = 0; h2 < 2; ++h2)
 #pragma unroll
-                        for (int c16 = 0; c16 < 8; ++c16)
-                            *reinterpret_cast<uint4 *>(vdst + h2 * kHalfBytes + row * 128 + c16 * 16) = make_uint4(0u, 0u, 0u, 0u);
+                            for (int c16 = 0; c16 < 8; ++c16)
+                                *reinterpret_cast<uint4 *>(vdst + h2 * kHalfBytes + row * 128 + c16 * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    fence_proxy_async_smem();
                 }
-                fence_proxy_async_smem();
-            }
 
-            // ---- the whole score row into registers (one TMEM read), masked entries become -inf
-            float sv[128];
-            {
-                uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
-                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
-                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
-                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
-                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
-                cp::tcgen05_wait_ld();
-            }
-            if (need_mask) {
+                // ---- the whole score row into registers (one TMEM read), masked entries become -inf
+                float sv[128];
+                {
+                    uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
+                    cp::tcgen05_wait_ld();
+                }
+                if (need_mask) {
 #pragma unroll
-                for (int i = 0; i < 128; ++i)
-                    if (key0 + i > lim || ((bad >> (i >> 4)) & 1)) sv[i] = -INFINITY;
-            }
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                    for (int i = 0; i < 128; ++i)
+                        if (key0 + i > lim || ((bad >> (i >> 4)) & 1)) sv[i] = -INFINITY;
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 128; i += 4) {
-                mx0 = fmaxf(mx0, sv[i]);
-                mx1 = fmaxf(mx1, sv[i + 1]);
-                mx2 = fmaxf(mx2, sv[i + 2]);
-                mx3 = fmaxf(mx3, sv[i + 3]);
-            }
-            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            const float m_tile = mx * p.scale_log2;  // scale > 0 on this path
-            // ---- lazy rescale: raise the reference max only when it is far behind
-            const bool raise = m_tile > m_run + kRescaleThreshold;  // also true for the first finite tile
-            if (__any_sync(0xffffffffu, raise)) {
-                const float m_new = raise ? m_tile : m_run;
-                const float alpha = (raise && m_run > -INFINITY) ? fast_exp2(m_run - m_new) : (raise ? 0.f : 1.f);
-                m_run = m_new;
-                l_run *= alpha;
-                if (j > 0) {  // O holds the sum over earlier tiles and no MMA touches it right now
+                for (int i = 0; i < 128; i += 4) {
+                    mx0 = fmaxf(mx0, sv[i]);
+                    mx1 = fmaxf(mx1, sv[i + 1]);
+                    mx2 = fmaxf(mx2, sv[i + 2]);
+                    mx3 = fmaxf(mx3, sv[i + 3]);
+                }
+                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                const float m_tile = mx * p.scale_log2;  // scale > 0 on this path
+                // ---- lazy rescale: raise the reference max only when it is far behind
+                const bool raise = m_tile > m_run + kRescaleThreshold;  // also true for the first finite tile
+                if (__any_sync(0xffffffffu, raise)) {
+                    const float m_new = raise ? m_tile : m_run;
+                    const float alpha = (raise && m_run > -INFINITY) ? fast_exp2(m_run - m_new) : (raise ? 0.f : 1.f);
+                    m_run = m_new;
+                    l_run *= alpha;
+                    if (j > 0) {  // O holds the sum over earlier tiles of this item and no MMA touches it right now
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        float ov[32];
-                        tmem_ld32(ov, t_o + 32 * cc);
+                        for (int cc = 0; cc < 4; ++cc) {
+                            float ov[32];
+                            tmem_ld32(ov, t_o + 32 * cc);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) ov[i] *= alpha;
-                        tmem_st32(t_o + 32 * cc, ov);
+                            for (int i = 0; i < 32; ++i) ov[i] *= alpha;
+                            tmem_st32(t_o + 32 * cc, ov);
+                        }
                     }
                 }
-            }
-            const float m_use = m_run > -INFINITY ? m_run : 0.f;
-            // ---- P = exp2(S*scale - m) (a masked -inf gives 0), row sum, bf16 pairs into the S columns
-            // P of the first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
-            float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
-            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
+                const float m_use = m_run > -INFINITY ? m_run : 0.f;
+                // ---- P = exp2(S*scale - m) (a masked -inf gives 0), row sum, bf16 pairs into the S columns
+                // P of the first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
+                float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                uint32_t pk[16];
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
-                    const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
-                    const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
-                    const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
-                    acc_a = __fadd2_rn(acc_a, pa);
-                    acc_b = __fadd2_rn(acc_b, pb);
-                    pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
-                    pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
+                    for (int i = 0; i < 32; i += 4) {
+                        const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
+                        const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
+                        const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
+                        const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+                        acc_a = __fadd2_rn(acc_a, pa);
+                        acc_b = __fadd2_rn(acc_b, pb);
+                        pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
+                        pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
+                    }
+                    cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
+                    if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
+                        cp::tcgen05_wait_st();
+                        fence_before();
+                        mbar_arrive(sh.bar(P_PART + x));
+                    }
                 }
-                cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
-                if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
-                    cp::tcgen05_wait_st();
-                    fence_before();
-                    mbar_arrive(sh.bar(P_PART + x));
-                }
+                l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
+                cp::tcgen05_wait_st();
+                fence_before();
+                mbar_arrive(sh.bar(P_READY + x));
             }
-            l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
-            cp::tcgen05_wait_st();
-            fence_before();
-            mbar_arrive(sh.bar(P_READY + x));
-        }
+            if (!ok) break;
 
-        // ---- epilogue: O / l -> bf16 -> this head's (now idle) Q tile in shared memory -> global.  A thread holds a
-        // whole row; writing it out directly would again touch 32 cache lines per instruction.  Each warp stages its
-        // 32 rows (16-byte pieces XOR-swizzled by row: no bank conflicts either way) and writes them back two rows
-        // per instruction, 256 contiguous bytes each.  Only the warp that wrote a row reads it: __syncwarp suffices.
-        if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)(n_tiles & 1), p.status, p.abort_word);
-        if (ok) {
-            fence_after();  // every MMA that read this Q tile has completed (the commit covers all earlier ones)
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            uint8_t *stage = sh.ptr + kOffQ + x * kTileBytes;
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                float ov[32];
-                tmem_ld32(ov, t_o + 32 * cc);
-#pragma unroll
-                for (int i = 0; i < 32; i += 8) {
-                    uint4 v;
-                    v.x = pack_bf16x2(ov[i] * inv, ov[i + 1] * inv);
-                    v.y = pack_bf16x2(ov[i + 2] * inv, ov[i + 3] * inv);
-                    v.z = pack_bf16x2(ov[i + 4] * inv, ov[i + 5] * inv);
-                    v.w = pack_bf16x2(ov[i + 6] * inv, ov[i + 7] * inv);
-                    const int piece = cc * 4 + (i >> 3);
-                    *reinterpret_cast<uint4 *>(stage + row * 256 + ((piece ^ (row & 15)) << 4)) = v;
-                }
+            // ---- write-out: O / l -> bf16 -> global.  The completion waited for here covers the item's last PV (and, if
+            // another item follows, its first QK^T: that wait is then not repeated).  The accumulator is read into
+            // registers in one go and handed back to the MMA warp at once; a thread holds a whole row, so the rows go
+            // through this warp's staging area (16-byte pieces XOR-swizzled by row) and leave as 128 contiguous bytes
+            // per row, four rows per instruction, one half of the channels at a time.
+            ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
+            if (!ok) break;
+            waited = true;
+            fence_after();
+            float ov[128];
+            {
+                uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(ov);
+                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_o);
+                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_o + 32);
+                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_o + 64);
+                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_o + 96);
+                cp::tcgen05_wait_ld();
             }
+            fence_before();
             __syncwarp();
-            const int piece = lane & 15;
-            __nv_bfloat16 *dst = p.out + ((size_t)(q0 + row0)) * row_stride + (size_t)head * kD + piece * 8;
+            if (lane == 0) mbar_arrive(sh.bar(O_FREE + x));
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            const int piece = lane & 7, sub = lane >> 3;
+            __nv_bfloat16 *dst = p.out + ((size_t)(it.q0 + it.row0)) * row_stride + (size_t)head * kD + piece * 8;
 #pragma unroll
-            for (int it = 0; it < 16; ++it) {
-                const int rr = wrow0 + 2 * it + (lane >> 4);
-                const uint4 v = *reinterpret_cast<const uint4 *>(stage + rr * 256 + ((piece ^ (rr & 15)) << 4));
-                if (rr < rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)rr * row_stride) = v;
+            for (int h2 = 0; h2 < 2; ++h2) {
+#pragma unroll
+                for (int i = 0; i < 64; i += 8) {
+                    uint4 v;
+                    v.x = pack_bf16x2(ov[64 * h2 + i] * inv, ov[64 * h2 + i + 1] * inv);
+                    v.y = pack_bf16x2(ov[64 * h2 + i + 2] * inv, ov[64 * h2 + i + 3] * inv);
+                    v.z = pack_bf16x2(ov[64 * h2 + i + 4] * inv, ov[64 * h2 + i + 5] * inv);
+                    v.w = pack_bf16x2(ov[64 * h2 + i + 6] * inv, ov[64 * h2 + i + 7] * inv);
+                    *reinterpret_cast<uint4 *>(stage + lane * 128 + (((i >> 3) ^ (lane & 7)) << 4)) = v;
+                }
+                __syncwarp();
+#pragma unroll
+                for (int r4 = 0; r4 < 8; ++r4) {
+                    const int lr = 4 * r4 + sub;  // row inside this warp's 32
+                    const uint4 v = *reinterpret_cast<const uint4 *>(stage + lr * 128 + ((piece ^ (lr & 7)) << 4));
+                    if (wrow0 + lr < it.rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)(wrow0 + lr) * row_stride + 64 * h2) = v;
+                }
+                __syncwarp();
             }
+            item_done();
         }
     }
 
@@ -507,17 +682,21 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     fence_before();
     __syncthreads();
     fence_after();
-    if (warp == 0 && *sh.abort_flag()) {
-        for (int j = max(0, n_tiles - kStages); j < n_tiles; ++j) {
-            (void)mbar_wait(sh.bar(K_FULL + j % kStages), (uint32_t)((j / kStages) & 1), 100000000ull);
-            (void)mbar_wait(sh.bar(V_FULL + j % kStages), (uint32_t)((j / kStages) & 1), 100000000ull);
+    if (*sh.abort_flag()) {
+        if (warp == 0 || warp == 2) {
+            const int FULL = warp == 2 ? V_FULL : K_FULL;
+            for (int j = max(0, tiles_issued - kStages); j < tiles_issued; ++j)
+                (void)mbar_wait(sh.bar(FULL + j % kStages), (uint32_t)((j / kStages) & 1), 100000000ull);
+        } else if (warp == 3 && tiles_issued > 0) {
+            for (int x = 0; x < 2; ++x) (void)mbar_wait(sh.bar(Q_FULL + x), (uint32_t)((tiles_issued - 1) & 1), 100000000ull);
         }
     }
     __syncthreads();
     if (warp == 2) cp::tcgen05_dealloc(cp::cta_group_1, tmem, 512);
 }
 
-static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillParams &p, int q_tiles, cudaStream_t stream) {
+static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillParams &p, const void *q, long long total_rows,
+                                      cudaStream_t stream) {
     static bool attr_set[64] = {false};
     const int dev = pool->desc.device;
     if (dev >= 64 || !attr_set[dev]) {
@@ -525,10 +704,14 @@ static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillPa
         if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_prefill_chunk: shared-memory attribute");
         if (dev < 64) attr_set[dev] = true;
     }
-    dim3 grid(q_tiles, pool->desc.num_q_heads / 2);
-    cudaError_t e0 = cudaMemsetAsync(p.abort_word, 0, sizeof(int), stream);
-    if (e0 != cudaSuccess) return cuda_fail(e0, "ekv_attn_prefill_chunk: clear abort word");
-    prefill_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(pool->kv_map[layer], p);
+    CUtensorMap qmap;
+    ekv_status_t st = encode_q_map(q, (uint64_t)total_rows, pool->desc.num_q_heads, kD, kBM, &qmap);
+    if (st != EKV_OK) return st;
+    const long long items = (long long)p.q_tiles * (pool->desc.num_q_heads / 2);
+    const int grid = (int)(items < pool->sm_count ? items : pool->sm_count);
+    cudaError_t e0 = cudaMemsetAsync(p.abort_word, 0, 2 * sizeof(int), stream);  // abort word + item counter
+    if (e0 != cudaSuccess) return cuda_fail(e0, "ekv_attn_prefill_chunk: clear abort word and item counter");
+    prefill_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(pool->kv_map[layer], qmap, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_prefill_chunk: launch");
     return EKV_OK;
