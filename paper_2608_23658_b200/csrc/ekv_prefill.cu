@@ -89,7 +89,7 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     p.q_tiles = (int)q_tiles;
     p.scale_log2 = scale * 1.4426950408889634f;
     const bool d128 = pool->desc.head_dim == 128;
-    if (kernel == K_TWO_HEAD) return tc::launch_prefill_tc(pool, layer, p, q, cu_q_lens_host[R], (cudaStream_t)stream);
+    if (kernel == K_TWO_HEAD) return tc::launch_prefill_tc(pool, layer, p, q, out, cu_q_lens_host[R], (cudaStream_t)stream);
     if (kernel == K_ONE_HEAD)
         return d128 ? tc1::launch_prefill_tc1<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream)
                     : tc1::launch_prefill_tc1<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);

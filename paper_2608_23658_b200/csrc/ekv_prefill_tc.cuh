@@ -76,7 +76,7 @@ static constexpr int kOffV = kOffK + kStages * kTileBytes;        // V stages
 static constexpr int kOffStage = kOffV + kStages * kTileBytes;    // write-out staging: 8 softmax warps x [32 rows][128 B]
 static constexpr int kStageBytes = 32 * 128;
 static constexpr int kOffBar = kOffStage + 8 * kStageBytes;       // mbarriers
-static constexpr int kSmemBytes = kOffBar + 256 + 1024;           // + alignment slack
+static constexpr int kSmemBytes = kOffBar + 512 + 1024;           // barriers, flags, item ring; + alignment slack
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
 // barrier slots (8 bytes each)
@@ -84,7 +84,7 @@ static constexpr int kItemRing = 4;   // item numbers posted ahead of the slowes
 static constexpr int kItemAhead = EKV_TC_ITEM_AHEAD;  // the scheduler keeps this many items posted beyond the one whose Q it loads
 enum Bar { Q_FULL = 0, Q_EMPTY = 2, K_FULL = 4, K_EMPTY = 6, V_FULL = 8, V_EMPTY = 10, S_READY = 12, P_READY = 14, P_PART = 16,
            O_FREE = 18, DRAIN = 20, ITEM_READY = 21, ITEM_DONE = ITEM_READY + kItemRing, NBAR = ITEM_DONE + 1 };
-static_assert(8 * NBAR + 32 + 4 * kItemRing <= 256, "barrier area");
+static_assert(8 * NBAR + 32 <= 256, "barrier area");
 
 // TMEM columns
 __device__ __forceinline__ constexpr uint32_t col_s(int x) { return 128u * (uint32_t)x; }
@@ -158,8 +158,8 @@ struct Shared {
     // key-tile count: the K producer may run two tiles ahead of the softmax warps (it only waits for the QK MMAs), so a
     // slot per STAGE would be overwritten before the softmax of the older tile has read it.
     __device__ __forceinline__ volatile int *bad_mask(int tile) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 16 + 4 * (tile & 3)); }
-    // item numbers posted by the scheduler: slot k % kItemRing holds the CTA's k-th item
-    __device__ __forceinline__ volatile int *item_slot(int k) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 32 + 4 * (k % kItemRing)); }
+    // items posted by the scheduler: slot k % kItemRing holds the CTA's k-th item
+    __device__ __forceinline__ uint4 *item_slot(int k) const { return (uint4 *)(ptr + kOffBar + 256 + 64 * (k % kItemRing)); }
 };
 
 // Bounded wait that also gives up as soon as another role has flagged an abort.
@@ -187,24 +187,28 @@ __device__ __forceinline__ bool wait_warp(const Shared &sh, int bar, uint32_t pa
     return __all_sync(0xffffffffu, wait_or_abort(sh, bar, parity, status, abort_word));
 }
 
-// The CTA's k-th item number, as posted by the scheduler (a number >= the item count ends the list); -1 if the wait
-// was given up.
-__device__ __forceinline__ int fetch_item(const Shared &sh, int k, unsigned *status, int *abort_word) {
-    if (!wait_warp(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1), status, abort_word)) return -1;
-    return *sh.item_slot(k);
-}
-
-// One work item, decoded the same way by every role.
+// One work item.  The scheduler decodes it (that takes dependent reads of device memory) and posts it in the ring;
+// every role then reads the same 48 bytes from shared memory.
 struct Item {
-    int req, q0, row0, rows_here, L, prefix, n_tiles, n_blocks, head0, g;
-    bool malformed;  // seq_len shorter than the chunk: rows are zero-filled, nothing is loaded or multiplied
+    int req;        // request
+    int qrow;       // row of the query / output tensor where the tile starts
+    int prow;       // absolute position (prefix + row inside the chunk) of the tile's first row
+    int rows_here;  // rows of the tile that belong to the request (1..128)
+    int L, n_tiles, n_blocks;  // keys of the request; key tiles / blocks any row of this tile may see
+    int head0, g;   // first of the two query heads; their kv-head
+    int spare;
+    int malformed;  // seq_len shorter than the chunk: rows are zero-filled, nothing is loaded or multiplied
+    int state;      // kItemWork, or kItemEnd: the list of this CTA ends here
 };
+static constexpr int kItemWork = 1, kItemEnd = 2;
+static_assert(sizeof(Item) == 48, "item slot");
 // Item order: head pairs are taken in groups of kPairGroup (0 = all pairs in one group); inside a group the query tiles
 // go from the heaviest (latest) to the lightest and every tile is listed for all pairs of the group before the next
 // tile.  One group per launch makes the list globally longest-first (the end of the launch is made of one-tile items,
 // so the CTAs finish together); smaller groups keep fewer kv-heads' K/V streaming through L2 at a time.
 static constexpr int kPairGroup = EKV_TC_PAIR_GROUP;
 __device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item &it) {
+    it.state = kItemWork;
     const int npairs = p.num_q_heads / 2;
     const int gp = kPairGroup > 0 ? kPairGroup : npairs;
     const int per_group = p.q_tiles * gp;
@@ -213,23 +217,39 @@ __device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item 
     const int rank = r / in_group;
     const int pair = grp * gp + (r - rank * in_group);
     const int tile_idx = p.q_tiles - 1 - rank;              // heaviest (latest) tiles first
-    int acc_tiles = 0, c_r = 0;
-    if (!find_request(p, tile_idx, kBM, it.req, acc_tiles, it.q0, c_r)) return false;
+    int acc_tiles = 0, c_r = 0, q0 = 0;
+    if (!find_request(p, tile_idx, kBM, it.req, acc_tiles, q0, c_r)) return false;
     it.head0 = 2 * pair;
     it.g = it.head0 / p.group;
-    it.row0 = (tile_idx - acc_tiles) * kBM;
+    const int row0 = (tile_idx - acc_tiles) * kBM;
     it.L = min(p.seq_lens[it.req], p.max_blocks * 16);
-    it.prefix = it.L - c_r;
-    it.rows_here = min(kBM, c_r - it.row0);
-    it.malformed = it.prefix < 0;
-    const int kv_end = min(it.L, it.prefix + it.row0 + it.rows_here);  // keys any row of this tile may see
+    const int prefix = it.L - c_r;
+    it.qrow = q0 + row0;
+    it.prow = prefix + row0;
+    it.rows_here = min(kBM, c_r - row0);
+    it.malformed = prefix < 0 ? 1 : 0;
+    it.spare = 0;
+    const int kv_end = min(it.L, it.prow + it.rows_here);  // keys any row of this tile may see
     it.n_tiles = (kv_end + kBN - 1) / kBN;
     it.n_blocks = (kv_end + 15) >> 4;
     return true;
 }
 
+// The CTA's k-th item as posted by the scheduler.  Returns 1 for an item to work on, 0 at the end of the list (or for
+// an item that names no request), -1 if the wait was given up.  A malformed item still counts as 1.
+__device__ __forceinline__ int fetch_item(const Shared &sh, int k, Item &it, unsigned *status, int *abort_word) {
+    if (!wait_warp(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1), status, abort_word)) return -1;
+    const uint4 *src = sh.item_slot(k);
+    const uint4 a = src[0], b = src[1], c = src[2];  // field by field: the struct stays in registers
+    it.req = (int)a.x, it.qrow = (int)a.y, it.prow = (int)a.z, it.rows_here = (int)a.w;
+    it.L = (int)b.x, it.spare = (int)b.y, it.n_tiles = (int)b.z, it.n_blocks = (int)b.w;
+    it.head0 = (int)c.x, it.g = (int)c.y, it.malformed = (int)c.z, it.state = (int)c.w;
+    return it.state == kItemWork ? 1 : 0;
+}
+
 __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_constant__ CUtensorMap kvmap,
                                                                  const __grid_constant__ CUtensorMap qmap,
+                                                                 const __grid_constant__ CUtensorMap omap,
                                                                  const PrefillParams p) {
     // a CTA of this launch already timed out: do not start more work (the flag lives in device memory and is
     // cleared by the launcher; the host-mapped status word is never polled here)
@@ -249,6 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     if (threadIdx.x == 0) {
         prefetch_tensormap(&kvmap);
         prefetch_tensormap(&qmap);
+        prefetch_tensormap(&omap);
         for (int x = 0; x < 2; ++x) {
             mbar_init(sh.bar(Q_FULL + x), 1);
             mbar_init(sh.bar(Q_EMPTY + x), 1);
@@ -293,10 +314,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         int t = 0;  // tiles issued so far (all items): stage t % kStages, use number t / kStages of that stage
         bool ok = true;
         for (int k = 0; ok; ++k) {
-            const int m = fetch_item(sh, k, p.status, p.abort_word);
-            if (m < 0 || m >= n_items) break;
             Item it;
-            if (!decode_item(p, m, it) || it.malformed) continue;
+            if (fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;
+            if (it.malformed) continue;
             const int *bt = p.block_tables + (size_t)it.req * p.max_blocks;
             auto load_id = [&](int j) {  // lane l: id of block 8j + l%8 (-1 past the end, -2 invalid)
                 int id = -1;
@@ -351,25 +371,30 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                     !wait_warp(sh, ITEM_DONE, (uint32_t)((posted - kItemRing) & 1), p.status, p.abort_word))
                     return false;
                 int m = 0;
+                if (lane == 0) m = atomicAdd(counter, 1);
+                m = __shfl_sync(0xffffffffu, m, 0);
+                Item it;
+                it.req = it.qrow = it.prow = it.rows_here = it.L = it.spare = it.n_tiles = it.n_blocks = it.head0 = it.g = it.malformed = 0;
+                if (m >= n_items || !decode_item(p, m, it)) it.state = kItemEnd;  // the end marker is posted once; nobody reads past it
+                drained = it.state == kItemEnd;
                 if (lane == 0) {
-                    m = atomicAdd(counter, 1);
-                    *sh.item_slot(posted) = m;
+                    uint4 *dst = sh.item_slot(posted);
+                    dst[0] = make_uint4((unsigned)it.req, (unsigned)it.qrow, (unsigned)it.prow, (unsigned)it.rows_here);
+                    dst[1] = make_uint4((unsigned)it.L, (unsigned)it.spare, (unsigned)it.n_tiles, (unsigned)it.n_blocks);
+                    dst[2] = make_uint4((unsigned)it.head0, (unsigned)it.g, (unsigned)it.malformed, (unsigned)it.state);
                     __threadfence_block();
                     mbar_arrive(sh.bar(ITEM_READY + posted % kItemRing));
                 }
-                m = __shfl_sync(0xffffffffu, m, 0);
-                drained = m >= n_items;  // the end marker is posted once; nobody reads past it
                 ++posted;
             }
             return true;
         };
         for (int k = 0; ok; ++k) {
             ok = post_until(k + kItemAhead);
-            if (!ok) break;
-            const int m = *sh.item_slot(k);  // posted by this warp (k < posted always holds here unless the list ended before k)
-            if (k >= posted || m >= n_items) break;
+            if (!ok || k >= posted) break;
             Item it;
-            if (!decode_item(p, m, it) || it.malformed) continue;
+            if (fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;  // posted by this warp: the wait passes at once
+            if (it.malformed) continue;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 // the previous item's last QK^T of this head has read the tile
@@ -380,7 +405,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 if (lane == 0) mbar_expect_tx(sh.bar(Q_FULL + x), kTileBytes);
                 __syncwarp();
                 if (lane < 2)  // rows past the end of the query tensor read as zero; rows past the request's chunk are never written out
-                    tma_load_3d(sh.base + kOffQ + x * kTileBytes + lane * kHalfBytes, &qmap, 64 * lane, it.head0 + x, it.q0 + it.row0,
+                    tma_load_3d(sh.base + kOffQ + x * kTileBytes + lane * kHalfBytes, &qmap, 64 * lane, it.head0 + x, it.qrow,
                                 sh.bar(Q_FULL + x));
             }
             if (ok) ++n;
@@ -410,15 +435,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         // key tile of the current one.
         int k_item = 0;
         bool list_ok = true, list_end = false;
-        Item cur, nxt;
+        struct Tiles { int n_tiles; } cur = {0}, nxt = {0};  // all this warp needs of an item: its number of key tiles
         bool have_cur = false, have_nxt = false;
-        auto advance = [&](Item &it, bool &have) {  // next well-formed item of this CTA, if any
+        auto advance = [&](Tiles &out, bool &have) {  // next well-formed item of this CTA, if any
             have = false;
             while (list_ok && !list_end && !have) {
-                const int m = fetch_item(sh, k_item++, p.status, p.abort_word);
-                if (m < 0) list_ok = false;
-                else if (m >= n_items) list_end = true;
-                else have = decode_item(p, m, it) && !it.malformed;
+                Item it;
+                const int st = fetch_item(sh, k_item++, it, p.status, p.abort_word);
+                if (st < 0) list_ok = false;
+                else if (st == 0) list_end = true;
+                else have = !it.malformed;
+                out.n_tiles = it.n_tiles;
             }
         };
         advance(cur, have_cur);
@@ -427,7 +454,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         int n = 0;   // items whose first QK^T has been issued
         bool ok = have_cur && list_ok;
         // first QK^T of an item: its Q tile of head x and (checked for head A) the K tile must have landed
-        auto first_qk = [&](int x, const Item &it) -> bool {
+        auto first_qk = [&](int x, const Tiles &it) -> bool {
             if (!wait_warp(sh, Q_FULL + x, (uint32_t)(n & 1), p.status, p.abort_word)) return false;
             if (x == 0 && !wait_warp(sh, K_FULL + t % kStages, (uint32_t)((t / kStages) & 1), p.status, p.abort_word)) return false;
             fence_after();
@@ -511,24 +538,20 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             if (lane == 0) mbar_arrive(sh.bar(ITEM_DONE));
         };
         for (int k = 0; ok; ++k) {
-            const int m = fetch_item(sh, k, p.status, p.abort_word);
-            if (m < 0 || m >= n_items) break;
             Item it;
-            if (!decode_item(p, m, it)) {
-                item_done();
-                continue;
-            }
-            const int head = it.head0 + x;
+            if (fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;
             if (it.malformed) {  // zero rows, latch
                 if (threadIdx.x == 128) atomicOr(p.status, EKV_DEV_FLAG_OOB);
                 for (int e = threadIdx.x - 128 - 128 * x; e < it.rows_here * kD; e += 128)
-                    p.out[((size_t)(it.q0 + it.row0 + e / kD)) * row_stride + (size_t)head * kD + e % kD] = __float2bfloat16_rn(0.f);
+                    p.out[((size_t)(it.qrow + e / kD)) * row_stride + (size_t)(it.head0 + x) * kD + e % kD] = __float2bfloat16_rn(0.f);
                 item_done();
                 continue;
             }
-            const int lim = it.prefix + it.row0 + min(row, it.rows_here - 1);  // last key this row may see
+            // only these four stay in registers over the key-tile loop; the write-out reads the rest from the ring again
+            const int lim = it.prow + min(row, it.rows_here - 1);  // last key this row may see
+            const int prow = it.prow, L = it.L, n_tiles = it.n_tiles;
             float m_run = -INFINITY, l_run = 0.f;
-            for (int j = 0; j < it.n_tiles; ++j, ++t) {
+            for (int j = 0; j < n_tiles; ++j, ++t) {
                 const int s = t % kStages;
                 if (!waited) ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
                 waited = false;
@@ -536,15 +559,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 fence_after();
                 const int key0 = j * kBN;
                 const int bad = *sh.bad_mask(t);
-                const bool need_mask = (key0 + kBN - 1 > it.prefix + it.row0) || bad != 0;
+                const bool need_mask = (key0 + kBN - 1 > prow) || bad != 0;
                 // keys of this tile that lie past the sequence end, or in a skipped block, may hold anything
                 // (unwritten slots): their V rows must not reach the tensor pipe, because 0 * NaN = NaN
-                const bool dirty_v = (key0 + kBN > it.L) || bad != 0;
+                const bool dirty_v = (key0 + kBN > L) || bad != 0;
                 if (dirty_v && x == 0) {
                     ok = wait_warp(sh, V_FULL + s, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
                     if (!ok) break;
                     uint8_t *vdst = sh.ptr + kOffV + s * kTileBytes;
-                    if ((key0 + row >= it.L) || ((bad >> (row >> 4)) & 1)) {  // thread `row` owns key row `row` of the tile
+                    if ((key0 + row >= L) || ((bad >> (row >> 4)) & 1)) {  // thread `row` owns key row `row` of the tile
 #pragma unroll
                         for (int h2 = 0; h2 < 2; ++h2)
 #pragma unroll
@@ -653,29 +676,48 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             if (lane == 0) mbar_arrive(sh.bar(O_FREE + x));
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
             const int piece = lane & 7, sub = lane >> 3;
-            __nv_bfloat16 *dst = p.out + ((size_t)(it.q0 + it.row0)) * row_stride + (size_t)head * kD + piece * 8;
+            // A warp whose 32 rows all belong to the request hands each staged half to the TMA unit (one instruction, the
+            // rows leave asynchronously); a warp at the ragged end of a chunk writes its valid rows itself.
+            const uint4 slot0 = sh.item_slot(k)[0], slot2 = sh.item_slot(k)[2];  // the slot is this item's until item_done()
+            const int qrow = (int)slot0.y, rows_here = (int)slot0.w, head = (int)slot2.x + x;
+            const bool by_tma = wrow0 + 32 <= rows_here;
+            __nv_bfloat16 *dst = p.out + (size_t)qrow * row_stride + (size_t)head * kD + piece * 8;
 #pragma unroll
             for (int h2 = 0; h2 < 2; ++h2) {
+                uint4 v[8];  // converted before the wait below, so that the arithmetic hides some of it
 #pragma unroll
                 for (int i = 0; i < 64; i += 8) {
-                    uint4 v;
-                    v.x = pack_bf16x2(ov[64 * h2 + i] * inv, ov[64 * h2 + i + 1] * inv);
-                    v.y = pack_bf16x2(ov[64 * h2 + i + 2] * inv, ov[64 * h2 + i + 3] * inv);
-                    v.z = pack_bf16x2(ov[64 * h2 + i + 4] * inv, ov[64 * h2 + i + 5] * inv);
-                    v.w = pack_bf16x2(ov[64 * h2 + i + 6] * inv, ov[64 * h2 + i + 7] * inv);
-                    *reinterpret_cast<uint4 *>(stage + lane * 128 + (((i >> 3) ^ (lane & 7)) << 4)) = v;
+                    v[i >> 3].x = pack_bf16x2(ov[64 * h2 + i] * inv, ov[64 * h2 + i + 1] * inv);
+                    v[i >> 3].y = pack_bf16x2(ov[64 * h2 + i + 2] * inv, ov[64 * h2 + i + 3] * inv);
+                    v[i >> 3].z = pack_bf16x2(ov[64 * h2 + i + 4] * inv, ov[64 * h2 + i + 5] * inv);
+                    v[i >> 3].w = pack_bf16x2(ov[64 * h2 + i + 6] * inv, ov[64 * h2 + i + 7] * inv);
                 }
+                if (lane == 0) bulk_wait_group_read_0();  // the staging area is no longer being read by an earlier store
                 __syncwarp();
 #pragma unroll
-                for (int r4 = 0; r4 < 8; ++r4) {
-                    const int lr = 4 * r4 + sub;  // row inside this warp's 32
-                    const uint4 v = *reinterpret_cast<const uint4 *>(stage + lr * 128 + ((piece ^ (lr & 7)) << 4));
-                    if (wrow0 + lr < it.rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)(wrow0 + lr) * row_stride + 64 * h2) = v;
+                for (int i = 0; i < 8; ++i)
+                    *reinterpret_cast<uint4 *>(stage + lane * 128 + ((i ^ (lane & 7)) << 4)) = v[i];  // = the 128-byte swizzle
+                if (by_tma) {
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_3d(&omap, smem_u32(stage), 64 * h2, head, qrow + wrow0);
+                        bulk_commit_group();
+                    }
+                } else {
+                    __syncwarp();
+#pragma unroll
+                    for (int r4 = 0; r4 < 8; ++r4) {
+                        const int lr = 4 * r4 + sub;  // row inside this warp's 32
+                        const uint4 v = *reinterpret_cast<const uint4 *>(stage + lr * 128 + ((piece ^ (lr & 7)) << 4));
+                        if (wrow0 + lr < rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)(wrow0 + lr) * row_stride + 64 * h2) = v;
+                    }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
             item_done();
         }
+        if (lane == 0) bulk_wait_group_0();  // every row this warp handed to the TMA unit has been written
     }
 
     // ---- teardown: everybody meets, copies in flight get a bounded chance to land, TMEM goes back
@@ -695,7 +737,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     if (warp == 2) cp::tcgen05_dealloc(cp::cta_group_1, tmem, 512);
 }
 
-static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillParams &p, const void *q, long long total_rows,
+static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillParams &p, const void *q, void *out, long long total_rows,
                                       cudaStream_t stream) {
     static bool attr_set[64] = {false};
     const int dev = pool->desc.device;
@@ -704,14 +746,15 @@ static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillPa
         if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_prefill_chunk: shared-memory attribute");
         if (dev < 64) attr_set[dev] = true;
     }
-    CUtensorMap qmap;
+    CUtensorMap qmap, omap;
     ekv_status_t st = encode_q_map(q, (uint64_t)total_rows, pool->desc.num_q_heads, kD, kBM, &qmap);
+    if (st == EKV_OK) st = encode_q_map(out, (uint64_t)total_rows, pool->desc.num_q_heads, kD, 32, &omap);  // same geometry, 32-row boxes
     if (st != EKV_OK) return st;
     const long long items = (long long)p.q_tiles * (pool->desc.num_q_heads / 2);
     const int grid = (int)(items < pool->sm_count ? items : pool->sm_count);
     cudaError_t e0 = cudaMemsetAsync(p.abort_word, 0, 2 * sizeof(int), stream);  // abort word + item counter
     if (e0 != cudaSuccess) return cuda_fail(e0, "ekv_attn_prefill_chunk: clear abort word and item counter");
-    prefill_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(pool->kv_map[layer], qmap, p);
+    prefill_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(pool->kv_map[layer], qmap, omap, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_prefill_chunk: launch");
     return EKV_OK;

@@ -5,14 +5,15 @@
 // it stages feeds two heads.  For a batch of SHORT prompts a CTA sees one to four key tiles, most of its life is
 // fixed cost (TMEM allocation, the Q tile, the first K/V tile, a strictly serial QK -> softmax -> PV -> write-out),
 // and with one CTA per SM nothing overlaps that.  This kernel halves the footprint -- 128 query rows of one head,
-// 256 TMEM columns (S 128 + O head_dim), about 97 KB of shared memory, 192 threads -- so that two CTAs share an SM
+// 256 TMEM columns (S 128 + O head_dim), about 97 KB of shared memory, 256 threads -- so that two CTAs share an SM
 // and one's fixed cost and softmax hide behind the other's MMAs.  It is also the tcgen05 path for head_dim 64 and
 // for odd query groups, which the two-head kernel cannot take.
 //
 //   warp 0        TMA producer of K and V tiles (16-token x 64-channel boxes gathered through the block table)
 //   warp 1        TMEM allocation; MMA issuer: S = Q K^T (both operands from shared memory) and
 //                 O += P V (P read from TMEM, V from shared memory, MN-major)
-//   warps 2-5     softmax, one thread per query row (= TMEM lane); same lazy-rescaling scheme as the two-head kernel
+//   warps 2-3     idle (they complete the utility warpgroup, see the register note below)
+//   warps 4-7     softmax, one thread per query row (= TMEM lane); same lazy-rescaling scheme as the two-head kernel
 //
 // One K and one V stage at head_dim 128 (two at 64): K(j+1) is loaded while softmax(j) and PV(j) run, V(j+1) while
 // QK(j+1) and softmax(j+1) run, and the other CTA of the SM fills the tensor pipe meanwhile.
@@ -27,16 +28,17 @@ using tc::fence_after;
 using tc::fence_before;
 
 static constexpr int kBM = 128, kBN = 128;
-static constexpr int kThreads = 192;
+static constexpr int kThreads = 256;
 static constexpr int kHalfBytes = 128 * 128;  // [128 rows][64 bf16], 128-byte swizzle
 static constexpr int kTmemCols = 256;
 static constexpr uint32_t kColS = 0, kColO = 128;
-// Registers: 192 threads x 168 (the cap two CTAs per SM leave) and no setmaxnreg.  The softmax code fits in 168, and
-// setmaxnreg must be executed by whole warpgroups (four consecutive warps starting at a multiple of four) that all ask
-// for the same thing: the utility warps 0-1 and the softmax warps 2-5 do not line up with that, and a warpgroup whose
-// warps disagree blocks without bound.
-static constexpr int kLaunchRegs = 168;
-static_assert(2 * kLaunchRegs * kThreads <= 65536, "two CTAs per SM");
+// Registers: two CTAs per SM leave 128 per thread at launch.  Warps 0-3 (producer, MMA issuer, two idle warps) form one
+// warpgroup and drop to kRegsUtil, warps 4-7 (softmax) form the other and rise to kRegsSoftmax.  setmaxnreg must be
+// executed by whole warpgroups (four consecutive warps from a multiple of four) that all ask for the same thing -- a
+// warpgroup whose warps disagree blocks without bound -- which is why the CTA carries two idle warps.
+static constexpr int kLaunchRegs = 128, kRegsUtil = 40, kRegsSoftmax = 216;
+static_assert(128 * kRegsUtil + 128 * kRegsSoftmax <= kLaunchRegs * kThreads, "setmaxnreg split exceeds the CTA's registers");
+static_assert(2 * kLaunchRegs * kThreads <= 65536 && kRegsUtil % 8 == 0 && kRegsSoftmax % 8 == 0, "two CTAs per SM");
 
 template <int D>
 struct Geo {
@@ -158,7 +160,8 @@ __global__ void __launch_bounds__(kThreads, 2) prefill_tc1_kernel(const __grid_c
     fence_after();
     const uint32_t tmem = *sh.tmem_slot();
 
-    if (warp < 2) {
+    if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         if (warp == 0) {
             // =========================== TMA producer: K(j), then V(j) ===========================
             const long long live = *p.live;
@@ -207,7 +210,7 @@ __global__ void __launch_bounds__(kThreads, 2) prefill_tc1_kernel(const __grid_c
                         tma_load_3d(tile_base + half * kHalfBytes + blk * 2048, &kvmap, 64 * half, row, my_id, sh.bar(FULL + s));
                 }
             }
-        } else {
+        } else if (warp == 1) {
             // =========================== MMA issuer ===========================
             const uint32_t q_lo = tc::desc_lo(sh.base + G::kOffQ, 16);
             const uint32_t k_lo0 = tc::desc_lo(sh.base + G::kOffK, 16), v_lo0 = tc::desc_lo(sh.base + G::kOffV, kHalfBytes);
@@ -260,6 +263,7 @@ __global__ void __launch_bounds__(kThreads, 2) prefill_tc1_kernel(const __grid_c
             (void)wait_warp<D>(sh, G::DRAIN, 0, p.status, p.abort_word);
         }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // =========================== softmax + epilogue ===========================
         const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31 belong to this warp
         const int wrow0 = quarter << 5;
