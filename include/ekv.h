@@ -308,6 +308,9 @@ EKV_API ekv_status_t ekv_hoststep_flush(ekv_hoststep_t *step, void *stream);
  * cu_q_lens: DEVICE int32 [R+1], non-decreasing, cu_q_lens[0] = 0.
  * cu_q_lens_host: HOST copy of the same R+1 values (used to size the launch without a sync).
  * Requests with seq_lens[r] < c_r are invalid (rows produce zeros, EKV_ERR_BLOCK_OOB is latched).
+ * Needs no workspace.  Calls on one pool may run at the same time on different streams; each call in flight
+ * holds one of 64 per-pool launch words (work counter of the persistent kernel), so more than 64 calls of one
+ * pool in flight at once are not supported.
  */
 EKV_API ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
                                     const int32_t *block_tables, int32_t max_blocks_per_seq,

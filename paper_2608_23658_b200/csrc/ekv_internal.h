@@ -12,6 +12,9 @@
 #define EKV_DEV_FLAG_OOB 1u
 #define EKV_DEV_FLAG_TIMEOUT 2u
 
+// Prefill launches of one pool that may be in flight at the same time (each owns one device word while it runs).
+#define EKV_LAUNCH_SLOTS 64
+
 struct ekv_pool {
     ekv_pool_desc_t desc;
     ekv_vmm_backend_t be;
@@ -37,7 +40,9 @@ struct ekv_pool {
     uint64_t layer_base(int layer) const { return fused ? va[0] + (uint64_t)layer * block_bytes : va[layer]; }
 
     // device state (absent when host_only)
-    long long *d_live;      // device words: [0] number of block ids kernels may dereference, [1] abort word
+    long long *d_live;      // device words: [0] number of block ids kernels may dereference; [1 .. kLaunchSlots] one word per
+                            // prefill launch in flight: low half = abort flag, high half = next item number
+    unsigned launch_seq;    // prefill launches so far (picks the slot)
     unsigned *h_status;     // pinned, host-mapped status word
     unsigned *d_status;     // its device alias
     unsigned long long *d_layer_base;  // device array: start address of every layer's range

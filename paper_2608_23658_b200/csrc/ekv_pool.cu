@@ -369,6 +369,7 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
     p->host_only = replaced;
     p->grown = false;
     p->live_limit = 0;
+    p->launch_seq = 0;
     p->d_live = nullptr;
     p->h_status = nullptr;
     p->d_status = nullptr;
@@ -436,8 +437,8 @@ ekv_status_t ekv_pool_create(const ekv_pool_desc_t *desc, ekv_pool_t **out) {
 
     p->live_limit = p->base_blocks + (p->grown ? p->elastic_blocks : 0);
     if (st == EKV_OK && !p->host_only) {
-        cudaError_t e = cudaMalloc((void **)&p->d_live, 2 * sizeof(long long));  // [0] live limit, [1] abort word
-        if (e == cudaSuccess) e = cudaMemset(p->d_live, 0, 2 * sizeof(long long));
+        cudaError_t e = cudaMalloc((void **)&p->d_live, (1 + EKV_LAUNCH_SLOTS) * sizeof(long long));  // [0] live limit, then launch words
+        if (e == cudaSuccess) e = cudaMemset(p->d_live, 0, (1 + EKV_LAUNCH_SLOTS) * sizeof(long long));
         if (e == cudaSuccess) e = cudaHostAlloc((void **)&p->h_status, sizeof(unsigned), cudaHostAllocMapped);
         if (e == cudaSuccess) {
             *p->h_status = 0;

@@ -80,7 +80,9 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     p.seq_lens = seq_lens;
     p.live = pool->d_live;
     p.status = pool->d_status;
-    p.abort_word = reinterpret_cast<int *>(pool->d_live + 1);
+    // every launch gets a device word of its own (abort flag + item counter), so that launches of one pool on different
+    // streams do not share them; the launcher clears the word on the stream before the kernel
+    p.abort_word = reinterpret_cast<int *>(pool->d_live + 1 + __atomic_fetch_add(&pool->launch_seq, 1u, __ATOMIC_RELAXED) % EKV_LAUNCH_SLOTS);
     p.max_blocks = max_blocks_per_seq;
     p.num_q_heads = pool->desc.num_q_heads;
     p.num_kv_heads = pool->desc.num_kv_heads;

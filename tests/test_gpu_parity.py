@@ -573,6 +573,37 @@ def test_prefill_edge_cases_bad_ids_empty_requests_negative_scale(prefill_kernel
         pool.close()
 
 
+def test_prefill_calls_in_flight_on_two_streams_keep_their_own_work_lists():
+    """Two chunked-prefill calls of one pool running at the same time (two streams, different requests): the persistent
+    kernel hands out its work items from a counter in device memory, and every launch must have its own."""
+    shape = I.LLAMA8B
+    case = Case(shape, [3000, 2500], 400, 97)
+    try:
+        scale = 1 / math.sqrt(shape.head_dim)
+        cus = [torch.tensor([0, 3000], dtype=torch.int32), torch.tensor([0, 2500], dtype=torch.int32)]
+        qs = [rand_q(98, 3000, shape).to(DEV), rand_q(99, 2500, shape).to(DEV)]
+        tabs = [case.d_tables[0:1].contiguous(), case.d_tables[1:2].contiguous()]
+        lens = [case.d_lengths[0:1].contiguous(), case.d_lengths[1:2].contiguous()]
+        dcu = [c.to(DEV) for c in cus]
+        alone = [case.pool.attn_prefill_chunk(0, qs[i], tabs[i], dcu[i], cus[i], lens[i], scale) for i in range(2)]
+        torch.cuda.synchronize()
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        outs = [torch.empty_like(q) for q in qs]
+        for rep in range(3):
+            for o in outs:
+                o.zero_()
+            torch.cuda.synchronize()
+            for i in range(2):
+                with torch.cuda.stream(streams[i]):
+                    case.pool.attn_prefill_chunk(0, qs[i], tabs[i], dcu[i], cus[i], lens[i], scale, out=outs[i], stream=streams[i])
+            torch.cuda.synchronize()
+            for i in range(2):
+                assert torch.equal(outs[i], alone[i]), f"call {i}, repetition {rep}"
+        assert case.pool.poll_status() == ekv.Status.OK
+    finally:
+        case.close()
+
+
 def test_prefill_kernel_families_agree_on_the_same_call():
     """The same call through each kernel family (pinned by its pool flag), each against the oracle and against the
     others."""
