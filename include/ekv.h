@@ -82,10 +82,10 @@ enum {
                                     until the next ekv_grow maps it again) */
     EKV_FUSED_RANGE = 1u << 2,   /* ekv_pool_create: ONE virtual range and two handles for all layers
                                     instead of one range and two handles per layer (see above) */
-    EKV_PREFILL_ONE_HEAD = 1u << 4, /* ekv_pool_create: ekv_attn_prefill_chunk on this pool always runs the
-                                    one-head-per-CTA tcgen05 kernel (normally chosen for head_dim 64, odd
-                                    query groups and batches of short chunks), so that it can be tested
-                                    and timed on any shape. */
+    EKV_PREFILL_ONE_HEAD = 1u << 4, /* ekv_pool_create: ekv_attn_prefill_chunk on this pool always runs a
+                                    tcgen05 kernel whose work item is ONE query head (normally chosen for
+                                    head_dim 64, odd query groups and batches of very short chunks), so
+                                    that it can be tested and timed on any shape. */
     EKV_PREFILL_TWO_HEAD = 1u << 5, /* ekv_pool_create: ekv_attn_prefill_chunk on this pool runs the two-head
                                     tcgen05 kernel whenever the shape allows it (head_dim 128, even query
                                     group, scale > 0), however short the chunks are. */

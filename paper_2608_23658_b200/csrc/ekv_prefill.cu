@@ -2,17 +2,18 @@
 // cu_q_lens (no device synchronisation) and dispatches the kernel for the pool's head_dim.
 #include "ekv_internal.h"
 #ifndef EKV_SHORT_CHUNK_ROWS
-#define EKV_SHORT_CHUNK_ROWS 0
+#define EKV_SHORT_CHUNK_ROWS 192
 #endif
 #include "ekv_prefill_mma.cuh"
 #include "ekv_prefill_tc.cuh"
 #include "ekv_prefill_tc1.cuh"
+#include "ekv_prefill_tcs.cuh"
 
 using namespace ekv;
 
-// Mean chunk length (query rows per request of the call) below which the one-head kernel takes a head_dim 128 /
-// even-group call.  0 = never: measured on 64 x 512 and 256 x 128 fresh prompts the two-head kernel is the faster
-// of the two (348 vs 472 us, 279 vs 316 us), so the one-head kernel serves only the shapes the other cannot take.
+// Mean chunk length (query rows per request of the call) below which a head_dim 128 / even-group call over short
+// sequences takes the two-slot kernel.  Measured, 32768 query tokens in one call: 256 x 128 fresh prompts 162 us (two-slot)
+// against 176 us (two-head); 64 x 512: 341 against 330; 16 x 2048: 771 against 614; 4 x 8192: 2.50 against 1.78 ms.
 static constexpr int kShortChunkMeanRows = EKV_SHORT_CHUNK_ROWS;
 
 extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
@@ -32,14 +33,16 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
         set_error("ekv_attn_prefill_chunk: cu_q_lens[0] must be 0");
         return EKV_ERR_INVALID;
     }
-    // Three kernels (scale > 0 unless stated):
-    //   two-head tcgen05 kernel  head_dim 128, even query group, long chunks: a CTA owns the SM and every K/V tile feeds two heads
-    //   one-head tcgen05 kernel  head_dim 64, odd query groups, and batches of short chunks (two CTAs per SM hide each
-    //                            other's fixed cost); EKV_PREFILL_ONE_HEAD / EKV_PREFILL_TWO_HEAD override the choice between the two
-    //   warp-level MMA kernel    non-positive scales, and every call on a pool created with EKV_PREFILL_WARP_MMA (which
-    //                            the tests use to check the kernel families against each other)
-    // Only chunk lengths are known on the host (the prefixes live in seq_lens on the device), so "short" is judged by
-    // the mean chunk length of the call.
+    // Kernels (scale > 0 unless stated):
+    //   two-head tcgen05 kernel   head_dim 128, even query group: a persistent CTA per SM, every K/V tile feeds two heads
+    //   two-slot tcgen05 kernel   head_dim 128, one head per work item, the CTA's two TMEM slots on their own clocks: odd
+    //                             query groups, and batches of chunks that are short AND provably over short sequences
+    //                             (the table is at most two key tiles wide), where it is the faster of the two
+    //   one-head tcgen05 kernel   head_dim 64 (one CTA per tile and head, two CTAs per SM)
+    //   warp-level MMA kernel     non-positive scales, and every call on a pool created with EKV_PREFILL_WARP_MMA (which
+    //                             the tests use to check the kernel families against each other)
+    // EKV_PREFILL_ONE_HEAD / EKV_PREFILL_TWO_HEAD override the choice between the first two.  Only chunk lengths and
+    // the table width are known on the host (the prefixes live in seq_lens on the device).
     const int group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     const uint32_t pf = pool->desc.flags;
     enum { K_TWO_HEAD, K_ONE_HEAD, K_WARP_MMA } kernel;
@@ -51,7 +54,8 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
         kernel = K_TWO_HEAD;
     } else {
         const long long total_rows = cu_q_lens_host[R];
-        kernel = total_rows < (long long)kShortChunkMeanRows * R ? K_ONE_HEAD : K_TWO_HEAD;
+        const bool tiny = max_blocks_per_seq * pool->desc.block_size <= 2 * tc::kBN && total_rows < (long long)kShortChunkMeanRows * R;
+        kernel = tiny ? K_ONE_HEAD : K_TWO_HEAD;
     }
     const int bm = kernel == K_WARP_MMA ? kPmBM : tc::kBM;
     PrefillParams p;
@@ -93,7 +97,7 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     const bool d128 = pool->desc.head_dim == 128;
     if (kernel == K_TWO_HEAD) return tc::launch_prefill_tc(pool, layer, p, q, out, cu_q_lens_host[R], (cudaStream_t)stream);
     if (kernel == K_ONE_HEAD)
-        return d128 ? tc1::launch_prefill_tc1<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream)
+        return d128 ? tcs::launch_prefill_tcs(pool, layer, p, q, out, cu_q_lens_host[R], (cudaStream_t)stream)
                     : tc1::launch_prefill_tc1<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);
     return d128 ? launch_prefill_mma<128>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream)
                 : launch_prefill_mma<64>(pool, layer, p, (int)q_tiles, (cudaStream_t)stream);

@@ -83,7 +83,7 @@ static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 static constexpr int kItemRing = 4;   // item numbers posted ahead of the slowest role
 static constexpr int kItemAhead = EKV_TC_ITEM_AHEAD;  // the scheduler keeps this many items posted beyond the one whose Q it loads
 enum Bar { Q_FULL = 0, Q_EMPTY = 2, K_FULL = 4, K_EMPTY = 6, V_FULL = 8, V_EMPTY = 10, S_READY = 12, P_READY = 14, P_PART = 16,
-           O_FREE = 18, DRAIN = 20, ITEM_READY = 21, ITEM_DONE = ITEM_READY + kItemRing, NBAR = ITEM_DONE + 1 };
+           O_FREE = 18, DRAIN = 20, ITEM_READY = 21, NBAR = ITEM_READY + kItemRing };
 static_assert(8 * NBAR + 32 <= 256, "barrier area");
 
 // TMEM columns
@@ -158,6 +158,10 @@ struct Shared {
     // key-tile count: the K producer may run two tiles ahead of the softmax warps (it only waits for the QK MMAs), so a
     // slot per STAGE would be overwritten before the softmax of the older tile has read it.
     __device__ __forceinline__ volatile int *bad_mask(int tile) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 16 + 4 * (tile & 3)); }
+    // Softmax warps that are through with an item (8 per item) are COUNTED, not signalled on an mbarrier: the scheduler
+    // looks at the count only when it needs a ring slot back, possibly a few items later, and a phase parity cannot tell
+    // "not yet" from "two phases ago".
+    __device__ __forceinline__ int *done_count() const { return (int *)(ptr + kOffBar + 8 * NBAR + 12); }
     // items posted by the scheduler: slot k % kItemRing holds the CTA's k-th item
     __device__ __forceinline__ uint4 *item_slot(int k) const { return (uint4 *)(ptr + kOffBar + 256 + 64 * (k % kItemRing)); }
 };
@@ -286,7 +290,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         }
         mbar_init(sh.bar(DRAIN), 1);
         for (int i = 0; i < kItemRing; ++i) mbar_init(sh.bar(ITEM_READY + i), 1);
-        mbar_init(sh.bar(ITEM_DONE), 8);
+        *sh.done_count() = 0;
         *sh.abort_flag() = 0;
         mbar_fence_init();
     }
@@ -367,9 +371,23 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         // k - kItemRing is written out: every role has long read it by then.
         auto post_until = [&](int upto) -> bool {
             while (posted <= upto && !drained) {
-                if (posted >= kItemRing &&
-                    !wait_warp(sh, ITEM_DONE, (uint32_t)((posted - kItemRing) & 1), p.status, p.abort_word))
-                    return false;
+                if (posted >= kItemRing) {  // the ring slot is free once all 8 softmax warps are through with item posted - kItemRing
+                    const int need = 8 * (posted - kItemRing + 1);
+                    const uint64_t t0 = global_timer_ns();
+                    bool got = false;
+                    for (uint32_t i = 0; !got; ++i) {
+                        got = *(volatile int *)sh.done_count() >= need;
+                        if (!got && (i & 31u) == 31u) {
+                            if (*sh.abort_flag()) return false;
+                            if (global_timer_ns() - t0 > 2000000000ull) {
+                                *sh.abort_flag() = 1;
+                                *(volatile int *)p.abort_word = 1;
+                                atomicOr(p.status, EKV_DEV_FLAG_TIMEOUT);
+                                return false;
+                            }
+                        }
+                    }
+                }
                 int m = 0;
                 if (lane == 0) m = atomicAdd(counter, 1);
                 m = __shfl_sync(0xffffffffu, m, 0);
@@ -535,7 +553,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         bool ok = true, waited = false;
         auto item_done = [&]() {  // this warp is through with the item: its slot in the ring may be reused
             __syncwarp();
-            if (lane == 0) mbar_arrive(sh.bar(ITEM_DONE));
+            if (lane == 0) {
+                __threadfence_block();
+                atomicAdd(sh.done_count(), 1);
+            }
         };
         for (int k = 0; ok; ++k) {
             Item it;
