@@ -1,20 +1,12 @@
 // ekv_attn_prefill_chunk: host entry point.  Validates, sizes the launch from the host copy of
 // cu_q_lens (no device synchronisation) and dispatches the kernel for the pool's head_dim.
 #include "ekv_internal.h"
-#ifndef EKV_SHORT_CHUNK_ROWS
-#define EKV_SHORT_CHUNK_ROWS 192
-#endif
 #include "ekv_prefill_mma.cuh"
 #include "ekv_prefill_tc.cuh"
 #include "ekv_prefill_tc1.cuh"
 #include "ekv_prefill_tcs.cuh"
 
 using namespace ekv;
-
-// Mean chunk length (query rows per request of the call) below which a head_dim 128 / even-group call over short
-// sequences takes the two-slot kernel.  Measured, 32768 query tokens in one call: 256 x 128 fresh prompts 162 us (two-slot)
-// against 176 us (two-head); 64 x 512: 341 against 330; 16 x 2048: 771 against 614; 4 x 8192: 2.50 against 1.78 ms.
-static constexpr int kShortChunkMeanRows = EKV_SHORT_CHUNK_ROWS;
 
 extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, const void *q, void *out,
                                                const int32_t *block_tables, int32_t max_blocks_per_seq,
@@ -34,15 +26,16 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
         return EKV_ERR_INVALID;
     }
     // Kernels (scale > 0 unless stated):
-    //   two-head tcgen05 kernel   head_dim 128, even query group: a persistent CTA per SM, every K/V tile feeds two heads
+    //   two-head tcgen05 kernel   head_dim 128, even query group: a persistent CTA per SM, every K/V tile feeds two heads.
+    //                             Measured, 32768 query tokens in one call: 256 x 128 fresh prompts 134 us against 161 us
+    //                             for the two-slot kernel; 64 x 512: 236 against 335; 16 x 2048: 545 against 770
     //   two-slot tcgen05 kernel   head_dim 128, one head per work item, the CTA's two TMEM slots on their own clocks: odd
-    //                             query groups, and batches of chunks that are short AND provably over short sequences
-    //                             (the table is at most two key tiles wide), where it is the faster of the two
+    //                             query groups
     //   one-head tcgen05 kernel   head_dim 64 (one CTA per tile and head, two CTAs per SM)
     //   warp-level MMA kernel     non-positive scales, and every call on a pool created with EKV_PREFILL_WARP_MMA (which
     //                             the tests use to check the kernel families against each other)
-    // EKV_PREFILL_ONE_HEAD / EKV_PREFILL_TWO_HEAD override the choice between the first two.  Only chunk lengths and
-    // the table width are known on the host (the prefixes live in seq_lens on the device).
+    // EKV_PREFILL_ONE_HEAD forces the one-head family on an even group; EKV_PREFILL_TWO_HEAD is what an even group at
+    // head_dim 128 gets anyway (kept so that a caller can say so).
     const int group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     const uint32_t pf = pool->desc.flags;
     enum { K_TWO_HEAD, K_ONE_HEAD, K_WARP_MMA } kernel;
@@ -50,12 +43,8 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
         kernel = K_WARP_MMA;
     } else if ((pf & EKV_PREFILL_ONE_HEAD) || pool->desc.head_dim != 128 || group % 2 != 0) {
         kernel = K_ONE_HEAD;
-    } else if (pf & EKV_PREFILL_TWO_HEAD) {
-        kernel = K_TWO_HEAD;
     } else {
-        const long long total_rows = cu_q_lens_host[R];
-        const bool tiny = max_blocks_per_seq * pool->desc.block_size <= 2 * tc::kBN && total_rows < (long long)kShortChunkMeanRows * R;
-        kernel = tiny ? K_ONE_HEAD : K_TWO_HEAD;
+        kernel = K_TWO_HEAD;
     }
     const int bm = kernel == K_WARP_MMA ? kPmBM : tc::kBM;
     PrefillParams p;

@@ -37,6 +37,8 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include <type_traits>
+
 #include "ekv_internal.h"
 #include "ekv_prefill_mma.cuh"  // PrefillParams
 #include "ptx.cuh"
@@ -103,9 +105,25 @@ static constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
     return ((addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
 }
-// These three are executed by the WHOLE (converged) issuing warp with warp-uniform operands; one lane, picked by
-// elect.sync inside the block, issues the instruction.  Written this way the operands can live in uniform
-// registers; wrapped in `if (lane == 0)` they are per-thread values that have to be moved over one by one.
+// One lane of the (converged) issuing warp, picked by elect.sync, issues a whole run of MMAs from inside a branch.
+// In that form the descriptors are 64-bit values that step by a compile-time constant and the compiler keeps them in
+// uniform registers: about three instructions per MMA.  (One elect per MMA with the operands put together inside the
+// asm block costs twice that, a plain `if (lane == 0)` nearly three times.  The issuing thread sets the pace of the CTA,
+// a 128x128x16 MMA occupies the tensor pipe for only 64 cycles, and the code has to stay small: see below.)
+__device__ __forceinline__ bool elect_one() {
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
+    return e != 0;
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// Older form, one elect per MMA (the one-head kernels still use it).
 template <bool kAcc>
 __device__ __forceinline__ void mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
     asm volatile(
@@ -166,29 +184,60 @@ struct Shared {
     __device__ __forceinline__ uint4 *item_slot(int k) const { return (uint4 *)(ptr + kOffBar + 256 + 64 * (k % kItemRing)); }
 };
 
-// Bounded wait that also gives up as soon as another role has flagged an abort.
-__device__ __forceinline__ bool wait_or_abort(const Shared &sh, int bar, uint32_t parity, unsigned *status, int *abort_word) {
-    const uint32_t b = sh.bar(bar);
-    if (mbar_try_wait(b, parity)) return true;
+// Bounded wait of a whole warp (every lane polls, all lanes agree on the outcome: the roles use warp-collective
+// instructions afterwards, so a warp must leave its loop as a whole).  It also gives up as soon as another role has
+// flagged an abort.  At the place that waits there is only one poll and a vote: a wait that is not over at once goes
+// on in ONE out-of-line copy of the polling loop.  (There are dozens of waits; with the loop, the clock and the
+// give-up path inlined at each, they were the largest part of the issuing warp's code, and the kernel has to stay
+// small enough for the instruction caches.)
+__device__ __noinline__ bool wait_slow(uint32_t b, uint32_t parity, volatile int *abort_flag, unsigned *status, int *abort_word) {
     const uint64_t t0 = global_timer_ns();
+    bool ok = false;
     for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(b, parity)) return true;
+        if (mbar_try_wait(b, parity)) {
+            ok = true;
+            break;
+        }
         if ((i & 31u) == 0u) {
-            if (*sh.abort_flag()) return false;
+            if (*abort_flag) break;
             if (global_timer_ns() - t0 > 2000000000ull) {
-                *sh.abort_flag() = 1;
+                *abort_flag = 1;
                 *(volatile int *)abort_word = 1;
                 atomicOr(status, EKV_DEV_FLAG_TIMEOUT);
-                return false;
+                break;
             }
         }
     }
+    return __all_sync(0xffffffffu, ok);
 }
-
-// Warp-uniform form: every lane polls, all lanes agree on the outcome (the roles use warp-collective
-// instructions afterwards, so a warp must leave its loop as a whole).
 __device__ __forceinline__ bool wait_warp(const Shared &sh, int bar, uint32_t parity, unsigned *status, int *abort_word) {
-    return __all_sync(0xffffffffu, wait_or_abort(sh, bar, parity, status, abort_word));
+    const uint32_t b = sh.bar(bar);
+    if (__all_sync(0xffffffffu, mbar_try_wait(b, parity))) return true;
+    return wait_slow(b, parity, sh.abort_flag(), status, abort_word);
+}
+// The same with the loop inline, for the softmax warps: a call does not fit their register budget, and they wait in few places.
+__device__ __forceinline__ bool wait_warp_inline(const Shared &sh, int bar, uint32_t parity, unsigned *status, int *abort_word) {
+    const uint32_t b = sh.bar(bar);
+    bool ok = mbar_try_wait(b, parity);
+    if (!ok) {
+        const uint64_t t0 = global_timer_ns();
+        for (uint32_t i = 1;; ++i) {
+            if (mbar_try_wait(b, parity)) {
+                ok = true;
+                break;
+            }
+            if ((i & 31u) == 0u) {
+                if (*sh.abort_flag()) break;
+                if (global_timer_ns() - t0 > 2000000000ull) {
+                    *sh.abort_flag() = 1;
+                    *(volatile int *)abort_word = 1;
+                    atomicOr(status, EKV_DEV_FLAG_TIMEOUT);
+                    break;
+                }
+            }
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
 }
 
 // One work item.  The scheduler decodes it (that takes dependent reads of device memory) and posts it in the ring;
@@ -241,8 +290,11 @@ __device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item 
 
 // The CTA's k-th item as posted by the scheduler.  Returns 1 for an item to work on, 0 at the end of the list (or for
 // an item that names no request), -1 if the wait was given up.  A malformed item still counts as 1.
+template <bool kInlineWait = false>
 __device__ __forceinline__ int fetch_item(const Shared &sh, int k, Item &it, unsigned *status, int *abort_word) {
-    if (!wait_warp(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1), status, abort_word)) return -1;
+    const bool got = kInlineWait ? wait_warp_inline(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1), status, abort_word)
+                                 : wait_warp(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1), status, abort_word);
+    if (!got) return -1;
     const uint4 *src = sh.item_slot(k);
     const uint4 a = src[0], b = src[1], c = src[2];  // field by field: the struct stays in registers
     it.req = (int)a.x, it.qrow = (int)a.y, it.prow = (int)a.z, it.rows_here = (int)a.w;
@@ -432,104 +484,103 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     } else {
         // =========================== MMA issuer ===========================
         // descriptor low words of the tile origins; stepping inside a tile adds a compile-time constant
-        const uint32_t q_lo[2] = {desc_lo(sh.base + kOffQ, 16), desc_lo(sh.base + kOffQ + kTileBytes, 16)};
+        const uint32_t q_lo0 = desc_lo(sh.base + kOffQ, 16);
         const uint32_t k_lo0 = desc_lo(sh.base + kOffK, 16), v_lo0 = desc_lo(sh.base + kOffV, kHalfBytes);
         auto issue_qk = [&](int x, int s) {  // S_x = Q_x K(s)^T
-            const uint32_t k_lo = k_lo0 + (uint32_t)s * (kTileBytes >> 4);
+            if (elect_one()) {
+                const uint64_t hi = (uint64_t)kDescHi << 32;
+                const uint64_t k_desc = hi | (k_lo0 + (uint32_t)s * (kTileBytes >> 4)), q_desc = hi | (q_lo0 + (uint32_t)x * (kTileBytes >> 4));
+                const uint32_t d = tmem + col_s(x);
 #pragma unroll
-            for (int k = 0; k < kD / 16; ++k) {
-                const uint32_t off = ((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4;
-                if (k == 0) mma_ss_lo<false>(tmem + col_s(x), q_lo[x] + off, k_lo + off, kIdescQK);
-                else mma_ss_lo<true>(tmem + col_s(x), q_lo[x] + off, k_lo + off, kIdescQK);
+                for (int k = 0; k < kD / 16; ++k) {
+                    const uint32_t off = ((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4;
+                    mma_ss(d, q_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
+                }
             }
+            __syncwarp();
         };
         auto issue_pv = [&](int x, int s, bool acc, int k0, int k1) {  // O_x (+)= P_x[:, 16k0:16k1] V(s)[16k0:16k1, :]
-            const uint32_t v_lo = v_lo0 + (uint32_t)s * (kTileBytes >> 4);
+            if (elect_one()) {
+                const uint64_t v_desc = ((uint64_t)kDescHi << 32) | (v_lo0 + (uint32_t)s * (kTileBytes >> 4));
+                const uint32_t d = tmem + col_o(x), a = tmem + col_s(x);
 #pragma unroll
-            for (int k = k0; k < k1; ++k)
-                mma_ts_lo_dyn(tmem + col_o(x), tmem + col_s(x) + 8 * k, v_lo + ((k * 2048) >> 4), kIdescPV, (acc || k > 0) ? 1u : 0u);
+                for (int k = k0; k < k1; ++k) mma_ts(d, a + 8 * k, v_desc + ((k * 2048) >> 4), kIdescPV, (acc || k > 0) ? 1u : 0u);
+            }
+            __syncwarp();
         };
-        // The item list of this CTA, one item ahead: the first QK^T of the next item is issued inside the last
-        // key tile of the current one.
+        // The item list of this CTA, one item ahead: the first QK^T of the next item is issued inside the last key tile of
+        // the current one.  The loop below is ONE copy of "PV of this key tile, then QK^T of the next key tile" for both
+        // heads, every kind of item boundary and the start of the list (an empty item with one tile that has no PV): this
+        // warp sets the pace of the CTA and shares an instruction cache with two softmax warps, so its code has to be
+        // small.  (Left to itself the compiler unrolls over the heads and clones the loop for each condition that does
+        // not change inside it; the values it would do that for pass through an empty asm statement.)
         int k_item = 0;
         bool list_ok = true, list_end = false;
-        struct Tiles { int n_tiles; } cur = {0}, nxt = {0};  // all this warp needs of an item: its number of key tiles
-        bool have_cur = false, have_nxt = false;
-        auto advance = [&](Tiles &out, bool &have) {  // next well-formed item of this CTA, if any
-            have = false;
-            while (list_ok && !list_end && !have) {
+        int cur_tiles = 1, nxt_tiles = 0;  // all this warp needs of an item: its number of key tiles
+        bool have_nxt = false;
+        int t = 0;   // key tiles whose QK^T (both heads) has been issued: the next QK^T reads K stage t % kStages
+        int tv = 0;  // key tiles whose PV has been issued
+        int n = 0;   // items whose first QK^T has been issued
+        int primed = 0;  // 0 while the "current item" is the empty one in front of the list
+        bool ok = true;
+        while (ok) {
+            have_nxt = false;  // next well-formed item of this CTA, if any
+            while (list_ok && !list_end && !have_nxt) {
                 Item it;
                 const int st = fetch_item(sh, k_item++, it, p.status, p.abort_word);
                 if (st < 0) list_ok = false;
                 else if (st == 0) list_end = true;
-                else have = !it.malformed;
-                out.n_tiles = it.n_tiles;
+                else have_nxt = !it.malformed;
+                nxt_tiles = it.n_tiles;
             }
-        };
-        advance(cur, have_cur);
-        int t = 0;   // key tiles whose QK^T (both heads) has been issued: the next QK^T reads K stage t % kStages
-        int tv = 0;  // key tiles whose PV has been issued
-        int n = 0;   // items whose first QK^T has been issued
-        bool ok = have_cur && list_ok;
-        // first QK^T of an item: its Q tile of head x and (checked for head A) the K tile must have landed
-        auto first_qk = [&](int x, const Tiles &it) -> bool {
-            if (!wait_warp(sh, Q_FULL + x, (uint32_t)(n & 1), p.status, p.abort_word)) return false;
-            if (x == 0 && !wait_warp(sh, K_FULL + t % kStages, (uint32_t)((t / kStages) & 1), p.status, p.abort_word)) return false;
-            fence_after();
-            issue_qk(x, t % kStages);
-            if (it.n_tiles == 1) mma_commit(sh.bar(Q_EMPTY + x));  // also the item's last QK^T of this head
-            return true;
-        };
-        if (ok) {
-            ok = first_qk(0, cur);
-            if (ok) mma_commit(sh.bar(S_READY + 0));
-            if (ok) ok = first_qk(1, cur);
-            if (ok) {
-                mma_commit(sh.bar(K_EMPTY + t % kStages));
-                mma_commit(sh.bar(S_READY + 1));
-                ++t;
-                ++n;
-            }
-        }
-        while (ok) {
-            advance(nxt, have_nxt);
-            if (!list_ok) break;
-            for (int j = 0; j < cur.n_tiles && ok; ++j, ++tv) {
+            if (!list_ok || (!primed && !have_nxt)) break;
+            int have_next = have_nxt ? 1 : 0, n_now = n, pv = primed;
+            asm volatile("" : "+r"(have_next), "+r"(n_now), "+r"(pv));
+#pragma unroll 1
+            for (int j = 0; j < cur_tiles && ok; ++j) {
                 const int s = tv % kStages;
-                const bool last = j + 1 == cur.n_tiles;
-                const bool more = !last || have_nxt;             // another key tile follows (this item's or the next one's)
-                const int s1 = t % kStages;                      // its stage
-                ok = wait_warp(sh, V_FULL + s, (uint32_t)((tv / kStages) & 1), p.status, p.abort_word);
-                if (ok && !last) ok = wait_warp(sh, K_FULL + s1, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
+                const bool last = j + 1 == cur_tiles;
+                const bool new_item = last && have_next;          // the next key tile opens the next item
+                const bool more = !last || have_next;             // another key tile follows (this item's or the next one's)
+                const int s1 = t % kStages;                       // its stage
+                // that tile is the last one of its item: its QK^T is the last reader of the item's Q tile
+                const bool next_closes = new_item ? nxt_tiles == 1 : j + 2 == cur_tiles;
+                if (pv) ok = wait_warp(sh, V_FULL + s, (uint32_t)((tv / kStages) & 1), p.status, p.abort_word);
 #pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    if (!ok) break;
-                    // O_x still holds the previous item's result until its write-out has read it
-                    if (j == 0 && n > 1) ok = wait_warp(sh, O_FREE + x, (uint32_t)((n - 2) & 1), p.status, p.abort_word);
-                    if (ok) ok = wait_warp(sh, P_PART + x, (uint32_t)(tv & 1), p.status, p.abort_word);
-                    if (!ok) break;
-                    fence_after();
-                    issue_pv(x, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
-                    ok = wait_warp(sh, P_READY + x, (uint32_t)(tv & 1), p.status, p.abort_word);
-                    if (!ok) break;
-                    fence_after();
-                    issue_pv(x, s, true, kPartSteps, kBN / 16);
-                    if (x == 1) mma_commit(sh.bar(V_EMPTY + s));
-                    if (!last) {
-                        issue_qk(x, s1);
-                        if (j + 2 == cur.n_tiles) mma_commit(sh.bar(Q_EMPTY + x));  // the item's last QK^T of this head
-                    } else if (have_nxt) {
-                        ok = first_qk(x, nxt);
+                for (int x = 0; x < 2 && ok; ++x) {
+                    if (pv) {
+                        // O_x still holds the previous item's result until its write-out has read it
+                        if (j == 0 && n_now > 1) ok = wait_warp(sh, O_FREE + x, (uint32_t)((n_now - 2) & 1), p.status, p.abort_word);
+                        if (ok) ok = wait_warp(sh, P_PART + x, (uint32_t)(tv & 1), p.status, p.abort_word);
                         if (!ok) break;
+                        fence_after();
+                        issue_pv(x, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
+                        ok = wait_warp(sh, P_READY + x, (uint32_t)(tv & 1), p.status, p.abort_word);
+                        if (!ok) break;
+                        fence_after();
+                        issue_pv(x, s, true, kPartSteps, kBN / 16);
+                        if (x == 1) mma_commit(sh.bar(V_EMPTY + s));
                     }
-                    if (x == 1 && more) mma_commit(sh.bar(K_EMPTY + s1));
-                    mma_commit(sh.bar(S_READY + x));  // scores of the next tile, and (after the last tile) O_x complete
+                    if (more) {
+                        // a new item: its Q tile of head x must have landed; head A also checks the K tile
+                        if (new_item) ok = wait_warp(sh, Q_FULL + x, (uint32_t)(n_now & 1), p.status, p.abort_word);
+                        if (ok && x == 0) ok = wait_warp(sh, K_FULL + s1, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
+                        if (!ok) break;
+                        fence_after();
+                        issue_qk(x, s1);
+                        if (next_closes) mma_commit(sh.bar(Q_EMPTY + x));
+                        if (x == 1) mma_commit(sh.bar(K_EMPTY + s1));
+                    }
+                    mma_commit(sh.bar(S_READY + x));  // scores of the next tile, and (after an item's last tile) O_x complete
                 }
-                if (ok && more) ++t;
-                if (ok && last && have_nxt) ++n;
+                if (!ok) break;
+                if (pv) ++tv;
+                if (more) ++t;
+                if (new_item) ++n;
             }
             if (!ok || !have_nxt) break;
-            cur = nxt;
+            cur_tiles = nxt_tiles;
+            primed = 1;
         }
         // every MMA this thread issued must be finished before TMEM is released
         mma_commit(sh.bar(DRAIN));
@@ -560,11 +611,14 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         };
         for (int k = 0; ok; ++k) {
             Item it;
-            if (fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;
+            if (fetch_item<true>(sh, k, it, p.status, p.abort_word) <= 0) break;
             if (it.malformed) {  // zero rows, latch
                 if (threadIdx.x == 128) atomicOr(p.status, EKV_DEV_FLAG_OOB);
-                for (int e = threadIdx.x - 128 - 128 * x; e < it.rows_here * kD; e += 128)
-                    p.out[((size_t)(it.qrow + e / kD)) * row_stride + (size_t)(it.head0 + x) * kD + e % kD] = __float2bfloat16_rn(0.f);
+                if (row < it.rows_here) {
+                    uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)(it.qrow + row) * row_stride + (size_t)(it.head0 + x) * kD);
+#pragma unroll 1
+                    for (int c = 0; c < kD / 8; ++c) o[c] = make_uint4(0u, 0u, 0u, 0u);
+                }
                 item_done();
                 continue;
             }
@@ -574,7 +628,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             float m_run = -INFINITY, l_run = 0.f;
             for (int j = 0; j < n_tiles; ++j, ++t) {
                 const int s = t % kStages;
-                if (!waited) ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
+                if (!waited) ok = wait_warp_inline(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
                 waited = false;
                 if (!ok) break;
                 fence_after();
@@ -585,89 +639,159 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 // (unwritten slots): their V rows must not reach the tensor pipe, because 0 * NaN = NaN
                 const bool dirty_v = (key0 + kBN > L) || bad != 0;
                 if (dirty_v && x == 0) {
-                    ok = wait_warp(sh, V_FULL + s, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
+                    ok = wait_warp_inline(sh, V_FULL + s, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
                     if (!ok) break;
                     uint8_t *vdst = sh.ptr + kOffV + s * kTileBytes;
                     if ((key0 + row >= L) || ((bad >> (row >> 4)) & 1)) {  // thread `row` owns key row `row` of the tile
-#pragma unroll
-                        for (int h2 = 0; h2 < 2; ++h2)
-#pragma unroll
-                            for (int c16 = 0; c16 < 8; ++c16)
-                                *reinterpret_cast<uint4 *>(vdst + h2 * kHalfBytes + row * 128 + c16 * 16) = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 1
+                        for (int c = 0; c < 16; ++c)  // rare: kept small
+                            *reinterpret_cast<uint4 *>(vdst + (c >> 3) * kHalfBytes + row * 128 + (c & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
                     }
                     fence_proxy_async_smem();
                 }
 
-                // ---- the whole score row into registers (one TMEM read), masked entries become -inf
-                float sv[128];
-                {
-                    uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
-                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
-                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
-                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
-                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
-                    cp::tcgen05_wait_ld();
-                }
-                if (need_mask) {
+                // Lazy rescale, shared by the two forms of a tile below: the reference max of a row is raised only when the
+                // tile's max is far above it (also for the row's first finite tile); O, if it holds anything yet, is then
+                // scaled in TMEM, 32 columns at a time (rare, so kept small rather than fast).
+                auto new_reference = [&](float m_tile) {
+                    const bool raise = m_tile > m_run + kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, raise)) {
+                        const float m_new = raise ? m_tile : m_run;
+                        const float alpha = (raise && m_run > -INFINITY) ? fast_exp2(m_run - m_new) : (raise ? 0.f : 1.f);
+                        m_run = m_new;
+                        l_run *= alpha;
+                        if (j > 0) {  // no MMA touches O_x right now
+#pragma unroll 1
+                            for (int cc = 0; cc < 4; ++cc) {
+                                float ov[32];
+                                tmem_ld32(ov, t_o + 32 * cc);
 #pragma unroll
-                    for (int i = 0; i < 128; ++i)
-                        if (key0 + i > lim || ((bad >> (i >> 4)) & 1)) sv[i] = -INFINITY;
-                }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                for (int i = 0; i < 128; i += 4) {
-                    mx0 = fmaxf(mx0, sv[i]);
-                    mx1 = fmaxf(mx1, sv[i + 1]);
-                    mx2 = fmaxf(mx2, sv[i + 2]);
-                    mx3 = fmaxf(mx3, sv[i + 3]);
-                }
-                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                const float m_tile = mx * p.scale_log2;  // scale > 0 on this path
-                // ---- lazy rescale: raise the reference max only when it is far behind
-                const bool raise = m_tile > m_run + kRescaleThreshold;  // also true for the first finite tile
-                if (__any_sync(0xffffffffu, raise)) {
-                    const float m_new = raise ? m_tile : m_run;
-                    const float alpha = (raise && m_run > -INFINITY) ? fast_exp2(m_run - m_new) : (raise ? 0.f : 1.f);
-                    m_run = m_new;
-                    l_run *= alpha;
-                    if (j > 0) {  // O holds the sum over earlier tiles of this item and no MMA touches it right now
-#pragma unroll
-                        for (int cc = 0; cc < 4; ++cc) {
-                            float ov[32];
-                            tmem_ld32(ov, t_o + 32 * cc);
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) ov[i] *= alpha;
-                            tmem_st32(t_o + 32 * cc, ov);
+                                for (int i = 0; i < 32; ++i) ov[i] *= alpha;
+                                tmem_st32(t_o + 32 * cc, ov);
+                            }
                         }
                     }
-                }
-                const float m_use = m_run > -INFINITY ? m_run : 0.f;
-                // ---- P = exp2(S*scale - m) (a masked -inf gives 0), row sum, bf16 pairs into the S columns
-                // P of the first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
-                float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
-                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
-                        const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
-                        const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
-                        const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
-                        acc_a = __fadd2_rn(acc_a, pa);
-                        acc_b = __fadd2_rn(acc_b, pb);
-                        pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
-                        pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
+                    return m_run > -INFINITY ? m_run : 0.f;
+                };
+                // The tile in two compiled forms: the plain one (nearly every tile of a long request; it holds nothing it
+                // does not need), and the one for a tile that the causal boundary cuts or that holds a block the table does
+                // not really name.  In the second, this row sees columns 0..rel of the tile; rel grows with the row, so a
+                // 32-column piece past the limit of the warp's last row holds nothing for the whole warp (no exponentials:
+                // P = 0), and inside a piece bit i of a word says that column i is hidden from this row.
+                if (!need_mask) {
+                    float sv[128];
+                    {
+                        uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
+                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
+                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
+                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
+                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
+                        cp::tcgen05_wait_ld();
                     }
-                    cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
-                    if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
-                        cp::tcgen05_wait_st();
-                        fence_before();
-                        mbar_arrive(sh.bar(P_PART + x));
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 128; i += 4) {
+                        mx0 = fmaxf(mx0, sv[i]);
+                        mx1 = fmaxf(mx1, sv[i + 1]);
+                        mx2 = fmaxf(mx2, sv[i + 2]);
+                        mx3 = fmaxf(mx3, sv[i + 3]);
                     }
+                    const float m_use = new_reference(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);  // scale > 0 on this path
+                    // ---- P = exp2(S*scale - m) (a hidden -inf gives 0), row sum, bf16 pairs into the S columns.  P of the
+                    // first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
+                    float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
+                    const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pk[16];
+                        {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4) {
+                                const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
+                                const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
+                                const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
+                                const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+                                acc_a = __fadd2_rn(acc_a, pa);
+                                acc_b = __fadd2_rn(acc_b, pb);
+                                pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
+                                pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
+                            }
+                        }
+                        cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
+                        if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
+                            cp::tcgen05_wait_st();
+                            fence_before();
+                            mbar_arrive(sh.bar(P_PART + x));
+                        }
+                    }
+                    l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
+                } else {
+                    float sv[128];
+                    {
+                        uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
+                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
+                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
+                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
+                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
+                        cp::tcgen05_wait_ld();
+                    }
+                    int rel_max = kBN;
+                    {
+                        const int rel = lim - key0;
+                        rel_max = __reduce_max_sync(0xffffffffu, rel);
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) {
+                            const int r = rel - 32 * cc;
+                            const unsigned past = r >= 31 ? 0u : (r < 0 ? 0xffffffffu : 0xfffffffeu << r);
+                            const unsigned b2 = (unsigned)bad >> (2 * cc);
+                            const unsigned hid = past | ((b2 & 1u) ? 0x0000ffffu : 0u) | ((b2 & 2u) ? 0xffff0000u : 0u);
+                            if (__any_sync(0xffffffffu, hid != 0u)) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) sv[32 * cc + i] = ((hid >> i) & 1u) ? -INFINITY : sv[32 * cc + i];
+                            }
+                        }
+                    }
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 128; i += 4) {
+                        mx0 = fmaxf(mx0, sv[i]);
+                        mx1 = fmaxf(mx1, sv[i + 1]);
+                        mx2 = fmaxf(mx2, sv[i + 2]);
+                        mx3 = fmaxf(mx3, sv[i + 3]);
+                    }
+                    const float m_use = new_reference(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);  // scale > 0 on this path
+                    // ---- P = exp2(S*scale - m) (a hidden -inf gives 0), row sum, bf16 pairs into the S columns.  P of the
+                    // first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
+                    float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
+                    const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pk[16];
+                        if (32 * cc > rel_max) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4) {
+                                const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
+                                const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
+                                const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
+                                const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+                                acc_a = __fadd2_rn(acc_a, pa);
+                                acc_b = __fadd2_rn(acc_b, pb);
+                                pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
+                                pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
+                            }
+                        }
+                        cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
+                        if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
+                            cp::tcgen05_wait_st();
+                            fence_before();
+                            mbar_arrive(sh.bar(P_PART + x));
+                        }
+                    }
+                    l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
                 }
-                l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
                 cp::tcgen05_wait_st();
                 fence_before();
                 mbar_arrive(sh.bar(P_READY + x));
@@ -679,22 +803,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             // registers in one go and handed back to the MMA warp at once; a thread holds a whole row, so the rows go
             // through this warp's staging area (16-byte pieces XOR-swizzled by row) and leave as 128 contiguous bytes
             // per row, four rows per instruction, one half of the channels at a time.
-            ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
+            ok = wait_warp_inline(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
             if (!ok) break;
             waited = true;
             fence_after();
-            float ov[128];
-            {
-                uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(ov);
-                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_o);
-                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_o + 32);
-                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_o + 64);
-                cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_o + 96);
-                cp::tcgen05_wait_ld();
-            }
-            fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(sh.bar(O_FREE + x));
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
             const int piece = lane & 7, sub = lane >> 3;
             // A warp whose 32 rows all belong to the request hands each staged half to the TMA unit (one instruction, the
@@ -703,15 +815,25 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             const int qrow = (int)slot0.y, rows_here = (int)slot0.w, head = (int)slot2.x + x;
             const bool by_tma = wrow0 + 32 <= rows_here;
             __nv_bfloat16 *dst = p.out + (size_t)qrow * row_stride + (size_t)head * kD + piece * 8;
-#pragma unroll
+            // One half of the channels at a time, as a loop (not unrolled: this code runs once per item).  The accumulator
+            // is handed back after the second half has been read; nothing waits for it sooner, because the next item's
+            // first PV needs the P that these same warps produce after this write-out.
+#pragma unroll 1
             for (int h2 = 0; h2 < 2; ++h2) {
-                uint4 v[8];  // converted before the wait below, so that the arithmetic hides some of it
+                float ov[64];
+                {
+                    uint32_t(&r)[64] = reinterpret_cast<uint32_t(&)[64]>(ov);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_o + 64 * h2);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_o + 64 * h2 + 32);
+                    cp::tcgen05_wait_ld();
+                }
+                uint4 v[8];
 #pragma unroll
                 for (int i = 0; i < 64; i += 8) {
-                    v[i >> 3].x = pack_bf16x2(ov[64 * h2 + i] * inv, ov[64 * h2 + i + 1] * inv);
-                    v[i >> 3].y = pack_bf16x2(ov[64 * h2 + i + 2] * inv, ov[64 * h2 + i + 3] * inv);
-                    v[i >> 3].z = pack_bf16x2(ov[64 * h2 + i + 4] * inv, ov[64 * h2 + i + 5] * inv);
-                    v[i >> 3].w = pack_bf16x2(ov[64 * h2 + i + 6] * inv, ov[64 * h2 + i + 7] * inv);
+                    v[i >> 3].x = pack_bf16x2(ov[i] * inv, ov[i + 1] * inv);
+                    v[i >> 3].y = pack_bf16x2(ov[i + 2] * inv, ov[i + 3] * inv);
+                    v[i >> 3].z = pack_bf16x2(ov[i + 4] * inv, ov[i + 5] * inv);
+                    v[i >> 3].w = pack_bf16x2(ov[i + 6] * inv, ov[i + 7] * inv);
                 }
                 if (lane == 0) bulk_wait_group_read_0();  // the staging area is no longer being read by an earlier store
                 __syncwarp();
@@ -727,15 +849,18 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                     }
                 } else {
                     __syncwarp();
-#pragma unroll
+#pragma unroll 1
                     for (int r4 = 0; r4 < 8; ++r4) {
                         const int lr = 4 * r4 + sub;  // row inside this warp's 32
-                        const uint4 v = *reinterpret_cast<const uint4 *>(stage + lr * 128 + ((piece ^ (lr & 7)) << 4));
-                        if (wrow0 + lr < rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)(wrow0 + lr) * row_stride + 64 * h2) = v;
+                        const uint4 w = *reinterpret_cast<const uint4 *>(stage + lr * 128 + ((piece ^ (lr & 7)) << 4));
+                        if (wrow0 + lr < rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)(wrow0 + lr) * row_stride + 64 * h2) = w;
                     }
                     __syncwarp();
                 }
             }
+            fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sh.bar(O_FREE + x));
             item_done();
         }
         if (lane == 0) bulk_wait_group_0();  // every row this warp handed to the TMA unit has been written
