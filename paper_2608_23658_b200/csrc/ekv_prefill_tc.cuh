@@ -673,125 +673,83 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                     }
                     return m_run > -INFINITY ? m_run : 0.f;
                 };
-                // The tile in two compiled forms: the plain one (nearly every tile of a long request; it holds nothing it
-                // does not need), and the one for a tile that the causal boundary cuts or that holds a block the table does
-                // not really name.  In the second, this row sees columns 0..rel of the tile; rel grows with the row, so a
-                // 32-column piece past the limit of the warp's last row holds nothing for the whole warp (no exponentials:
-                // P = 0), and inside a piece bit i of a word says that column i is hidden from this row.
-                if (!need_mask) {
-                    float sv[128];
-                    {
-                        uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
-                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
-                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
-                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
-                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
-                        cp::tcgen05_wait_ld();
-                    }
-                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                    for (int i = 0; i < 128; i += 4) {
-                        mx0 = fmaxf(mx0, sv[i]);
-                        mx1 = fmaxf(mx1, sv[i + 1]);
-                        mx2 = fmaxf(mx2, sv[i + 2]);
-                        mx3 = fmaxf(mx3, sv[i + 3]);
-                    }
-                    const float m_use = new_reference(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);  // scale > 0 on this path
-                    // ---- P = exp2(S*scale - m) (a hidden -inf gives 0), row sum, bf16 pairs into the S columns.  P of the
-                    // first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
-                    float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
-                    const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
-#pragma unroll
+                // A tile that the causal boundary cuts (or that holds a block the table does not really name) first gets
+                // its hidden scores overwritten with -inf IN TMEM, by a small loop over 32-column pieces, and then goes
+                // through the same code as every other tile.  This row sees columns 0..rel of the tile and rel grows with
+                // the row, so a piece is left alone if the warp's first row sees all of it, and is -inf for every row of
+                // the warp if the last row sees none of it.  (Such a tile comes once per item: for a long request its speed
+                // does not matter, and for a batch of short ones the SIZE of the code does -- their items walk through all
+                // of the softmax code every few thousand cycles, and what does not fit the instruction cache of the SM's
+                // quarter is fetched again for every item.)
+                if (need_mask) {
+                    const int rel = lim - key0;
+                    const int rel_min = __reduce_min_sync(0xffffffffu, rel), rel_max = __reduce_max_sync(0xffffffffu, rel);
+#pragma unroll 1
                     for (int cc = 0; cc < 4; ++cc) {
-                        uint32_t pk[16];
-                        {
-#pragma unroll
-                            for (int i = 0; i < 32; i += 4) {
-                                const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
-                                const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
-                                const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
-                                const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
-                                acc_a = __fadd2_rn(acc_a, pa);
-                                acc_b = __fadd2_rn(acc_b, pb);
-                                pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
-                                pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
-                            }
-                        }
-                        cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
-                        if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
-                            cp::tcgen05_wait_st();
-                            fence_before();
-                            mbar_arrive(sh.bar(P_PART + x));
-                        }
-                    }
-                    l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
-                } else {
-                    float sv[128];
-                    {
-                        uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
-                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
-                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
-                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
-                        cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
-                        cp::tcgen05_wait_ld();
-                    }
-                    int rel_max = kBN;
-                    {
-                        const int rel = lim - key0;
-                        rel_max = __reduce_max_sync(0xffffffffu, rel);
-#pragma unroll
-                        for (int cc = 0; cc < 4; ++cc) {
-                            const int r = rel - 32 * cc;
-                            const unsigned past = r >= 31 ? 0u : (r < 0 ? 0xffffffffu : 0xfffffffeu << r);
-                            const unsigned b2 = (unsigned)bad >> (2 * cc);
-                            const unsigned hid = past | ((b2 & 1u) ? 0x0000ffffu : 0u) | ((b2 & 2u) ? 0xffff0000u : 0u);
-                            if (__any_sync(0xffffffffu, hid != 0u)) {
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) sv[32 * cc + i] = ((hid >> i) & 1u) ? -INFINITY : sv[32 * cc + i];
-                            }
-                        }
-                    }
-                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                    for (int i = 0; i < 128; i += 4) {
-                        mx0 = fmaxf(mx0, sv[i]);
-                        mx1 = fmaxf(mx1, sv[i + 1]);
-                        mx2 = fmaxf(mx2, sv[i + 2]);
-                        mx3 = fmaxf(mx3, sv[i + 3]);
-                    }
-                    const float m_use = new_reference(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);  // scale > 0 on this path
-                    // ---- P = exp2(S*scale - m) (a hidden -inf gives 0), row sum, bf16 pairs into the S columns.  P of the
-                    // first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
-                    float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
-                    const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        uint32_t pk[16];
+                        const unsigned b2 = ((unsigned)bad >> (2 * cc)) & 3u;
+                        if (32 * cc + 31 <= rel_min && b2 == 0u) continue;
+                        const int r = rel - 32 * cc;
+                        const unsigned past = r >= 31 ? 0u : (r < 0 ? 0xffffffffu : 0xfffffffeu << r);
+                        const unsigned hid = past | ((b2 & 1u) ? 0x0000ffffu : 0u) | ((b2 & 2u) ? 0xffff0000u : 0u);
+                        float v[32];
                         if (32 * cc > rel_max) {
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+                            for (int i = 0; i < 32; ++i) v[i] = -INFINITY;
                         } else {
+                            tmem_ld32(v, t_s + 32 * cc);
 #pragma unroll
-                            for (int i = 0; i < 32; i += 4) {
-                                const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
-                                const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
-                                const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
-                                const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
-                                acc_a = __fadd2_rn(acc_a, pa);
-                                acc_b = __fadd2_rn(acc_b, pb);
-                                pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
-                                pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
-                            }
+                            for (int i = 0; i < 32; ++i) v[i] = ((hid >> i) & 1u) ? -INFINITY : v[i];
                         }
-                        cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
-                        if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
-                            cp::tcgen05_wait_st();
-                            fence_before();
-                            mbar_arrive(sh.bar(P_PART + x));
+                        tmem_st32(t_s + 32 * cc, v);
+                    }
+                    cp::tcgen05_wait_st();
+                }
+                float sv[128];
+                {
+                    uint32_t(&r)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_s);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_s + 32);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[64]), t_s + 64);
+                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[96]), t_s + 96);
+                    cp::tcgen05_wait_ld();
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 128; i += 4) {
+                    mx0 = fmaxf(mx0, sv[i]);
+                    mx1 = fmaxf(mx1, sv[i + 1]);
+                    mx2 = fmaxf(mx2, sv[i + 2]);
+                    mx3 = fmaxf(mx3, sv[i + 3]);
+                }
+                const float m_use = new_reference(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);  // scale > 0 on this path
+                // ---- P = exp2(S*scale - m) (a hidden -inf gives 0), row sum, bf16 pairs into the S columns.  P of the
+                // first 96 keys is published early so the PV MMA overlaps the last quarter of this loop.
+                float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_use, -m_use);
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t pk[16];
+                    {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            const float2 xa = __ffma2_rn(make_float2(sv[32 * cc + i], sv[32 * cc + i + 1]), sc2, nm2);
+                            const float2 xb = __ffma2_rn(make_float2(sv[32 * cc + i + 2], sv[32 * cc + i + 3]), sc2, nm2);
+                            const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
+                            const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+                            acc_a = __fadd2_rn(acc_a, pa);
+                            acc_b = __fadd2_rn(acc_b, pb);
+                            pk[i >> 1] = pack_bf16x2(pa.x, pa.y);
+                            pk[(i >> 1) + 1] = pack_bf16x2(pb.x, pb.y);
                         }
                     }
-                    l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
+                    cp::tcgen05_st_32x32b(t_s + 16 * cc, pk);
+                    if (cc == kPartSteps / 2 - 1) {  // 96 keys stored
+                        cp::tcgen05_wait_st();
+                        fence_before();
+                        mbar_arrive(sh.bar(P_PART + x));
+                    }
                 }
+                l_run += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
                 cp::tcgen05_wait_st();
                 fence_before();
                 mbar_arrive(sh.bar(P_READY + x));
