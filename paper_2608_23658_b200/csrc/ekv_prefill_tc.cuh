@@ -24,8 +24,19 @@
 //                 S_A S_B O_A O_B, P aliases S)
 //   warp 3        item scheduler; TMA producer of the two Q tiles of an item (one tensor map over
 //                 the query tensor)
-//   warps 4-7     softmax of head A: one thread per query row (= TMEM lane); write-out of head A
-//   warps 8-11    softmax and write-out of head B
+//   warps 4-7     softmax of head A: one thread per query row (= TMEM lane)
+//   warps 8-11    softmax of head B
+//   warps 12-15   write-out of both heads (O / l -> bf16 -> global, TMA stores), one warp per quarter
+//                 of the TMEM lanes: the softmax warps go from an item's last key tile straight to
+//                 the next item's first
+//
+// The code is kept SMALL on purpose.  Each quarter of the SM has an instruction cache of about 32 KB
+// for its four warps (measured: straight-line code runs at 1.0-1.2 cycles per instruction up to that
+// footprint and at 2.7 beyond it).  An item of a short request is a few key tiles long, so every role
+// walks through all of its code every few thousand cycles; what does not fit is fetched again for
+// every item.  Hence one copy of the MMA issuing loop, waits whose slow path is one out-of-line
+// function, rare paths as small loops, and one copy of the softmax code (a tile cut by the causal
+// boundary has its hidden scores set to -inf in TMEM first).
 //
 // Softmax is online in the exp2 domain with LAZY rescaling: the running reference max of a row is
 // only raised (and O, l rescaled in TMEM) when a tile's max exceeds it by more than 2^8, so P stays
@@ -61,31 +72,32 @@ static constexpr int kD = 128;           // head_dim
 static constexpr int kHalfBytes = 128 * 128;           // [128 rows][64 bf16]: one swizzled half tile
 static constexpr int kTileBytes = 2 * kHalfBytes;       // 32 KiB: a Q, K or V tile
 static constexpr int kStages = 2;
-static constexpr int kThreads = 384;
+static constexpr int kThreads = 512;
 static constexpr float kRescaleThreshold = 8.f;        // log2 units
-// Register re-partition (setmaxnreg): the CTA owns kLaunchRegs x kThreads registers.  Warps 0-3 drop to
-// kRegsUtil, warps 4-11 rise to kRegsSoftmax.  The raise BLOCKS until the pool has the registers, so
-// the split must fit the CTA's own allocation exactly -- nothing else bounds that wait -- and every
-// warpgroup (four consecutive warps from a multiple of four) must ask for the same thing.
-static constexpr int kLaunchRegs = 168, kRegsUtil = 72, kRegsSoftmax = 216;
-static_assert(128 * kRegsUtil + 256 * kRegsSoftmax <= kLaunchRegs * kThreads, "setmaxnreg split exceeds the CTA's registers");
-static_assert(kLaunchRegs * kThreads <= 65536 && kRegsUtil % 8 == 0 && kRegsSoftmax % 8 == 0, "register split");
+// Register re-partition (setmaxnreg): the CTA owns kLaunchRegs x kThreads registers.  Warps 0-3 (utility) and 12-15
+// (write-out) drop to kRegsUtil / kRegsOut, warps 4-11 (softmax) rise to kRegsSoftmax.  The raise BLOCKS until the pool
+// has the registers, so the split must fit the CTA's own allocation exactly -- nothing else bounds that wait -- and
+// every warpgroup (four consecutive warps from a multiple of four) must ask for the same thing.
+static constexpr int kLaunchRegs = 128, kRegsUtil = 72, kRegsSoftmax = 184, kRegsOut = 72;
+static_assert(128 * (kRegsUtil + kRegsOut) + 256 * kRegsSoftmax <= kLaunchRegs * kThreads, "setmaxnreg split exceeds the CTA's registers");
+static_assert(kLaunchRegs * kThreads <= 65536 && kRegsUtil % 8 == 0 && kRegsSoftmax % 8 == 0 && kRegsOut % 8 == 0, "register split");
 
 // shared-memory map (offsets from the 1024-byte aligned base)
 static constexpr int kOffQ = 0;                                   // Q_A, Q_B
 static constexpr int kOffK = kOffQ + 2 * kTileBytes;              // K stages
 static constexpr int kOffV = kOffK + kStages * kTileBytes;        // V stages
-static constexpr int kOffStage = kOffV + kStages * kTileBytes;    // write-out staging: 8 softmax warps x [32 rows][128 B]
+static constexpr int kOffStage = kOffV + kStages * kTileBytes;    // write-out staging: 4 write-out warps x 2 x [32 rows][128 B]
 static constexpr int kStageBytes = 32 * 128;
 static constexpr int kOffBar = kOffStage + 8 * kStageBytes;       // mbarriers
-static constexpr int kSmemBytes = kOffBar + 512 + 1024;           // barriers, flags, item ring; + alignment slack
+static constexpr int kOffInvL = kOffBar + 512;                     // 1 / row sum of the finished item: [2 heads][128 rows] floats
+static constexpr int kSmemBytes = kOffInvL + 1024 + 1024;         // barriers, flags, item ring; row sums; + alignment slack
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
 // barrier slots (8 bytes each)
 static constexpr int kItemRing = 4;   // item numbers posted ahead of the slowest role
 static constexpr int kItemAhead = EKV_TC_ITEM_AHEAD;  // the scheduler keeps this many items posted beyond the one whose Q it loads
 enum Bar { Q_FULL = 0, Q_EMPTY = 2, K_FULL = 4, K_EMPTY = 6, V_FULL = 8, V_EMPTY = 10, S_READY = 12, P_READY = 14, P_PART = 16,
-           O_FREE = 18, DRAIN = 20, ITEM_READY = 21, NBAR = ITEM_READY + kItemRing };
+           O_FREE = 18, DRAIN = 20, L_READY = 21, ITEM_READY = 23, NBAR = ITEM_READY + kItemRing };
 static_assert(8 * NBAR + 32 <= 256, "barrier area");
 
 // TMEM columns
@@ -176,10 +188,11 @@ struct Shared {
     // key-tile count: the K producer may run two tiles ahead of the softmax warps (it only waits for the QK MMAs), so a
     // slot per STAGE would be overwritten before the softmax of the older tile has read it.
     __device__ __forceinline__ volatile int *bad_mask(int tile) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 16 + 4 * (tile & 3)); }
-    // Softmax warps that are through with an item (8 per item) are COUNTED, not signalled on an mbarrier: the scheduler
+    // Softmax and write-out warps that are through with an item (12 per item) are COUNTED, not signalled on an mbarrier: the scheduler
     // looks at the count only when it needs a ring slot back, possibly a few items later, and a phase parity cannot tell
     // "not yet" from "two phases ago".
     __device__ __forceinline__ int *done_count() const { return (int *)(ptr + kOffBar + 8 * NBAR + 12); }
+    __device__ __forceinline__ float *inv_l(int x) const { return (float *)(ptr + kOffInvL) + 128 * x; }
     // items posted by the scheduler: slot k % kItemRing holds the CTA's k-th item
     __device__ __forceinline__ uint4 *item_slot(int k) const { return (uint4 *)(ptr + kOffBar + 256 + 64 * (k % kItemRing)); }
 };
@@ -333,6 +346,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             mbar_init(sh.bar(P_READY + x), 128);
             mbar_init(sh.bar(P_PART + x), 128);
             mbar_init(sh.bar(O_FREE + x), 4);
+            mbar_init(sh.bar(L_READY + x), 128);
         }
         for (int s = 0; s < kStages; ++s) {
             mbar_init(sh.bar(K_FULL + s), 1);
@@ -423,12 +437,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         // k - kItemRing is written out: every role has long read it by then.
         auto post_until = [&](int upto) -> bool {
             while (posted <= upto && !drained) {
-                if (posted >= kItemRing) {  // the ring slot is free once all 8 softmax warps are through with item posted - kItemRing
-                    const int need = 8 * (posted - kItemRing + 1);
+                if (posted >= kItemRing) {  // the ring slot is free once the 8 softmax and 4 write-out warps are through with item posted - kItemRing
+                    const int need = 12 * (posted - kItemRing + 1);
                     const uint64_t t0 = global_timer_ns();
                     bool got = false;
                     for (uint32_t i = 0; !got; ++i) {
                         got = *(volatile int *)sh.done_count() >= need;
+                        if (!got) __nanosleep(100);  // nothing urgent: leave the issue slots to the softmax warp next door
                         if (!got && (i & 31u) == 31u) {
                             if (*sh.abort_flag()) return false;
                             if (global_timer_ns() - t0 > 2000000000ull) {
@@ -586,22 +601,22 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         mma_commit(sh.bar(DRAIN));
         (void)wait_warp(sh, DRAIN, 0, p.status, p.abort_word);
     }
-    } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-        // =========================== softmax + write-out ===========================
+    } else if (warp < 12) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 184;");
+        // =========================== softmax ===========================
         const int x = (warp - 4) >> 2;                  // 0 = head A, 1 = head B
         const int wrow0 = (warp & 3) << 5;               // this warp's 32 rows of the tile = its TMEM lanes
         const int row = wrow0 | lane;                    // query row in the tile = TMEM lane
         const uint32_t lane_base = (uint32_t)wrow0 << 16;
         const uint32_t t_s = tmem + lane_base + col_s(x);
         const uint32_t t_o = tmem + lane_base + col_o(x);
-        uint8_t *stage = sh.ptr + kOffStage + (warp - 4) * kStageBytes;
 
         // S_READY_x completes once per key tile of the CTA (all items), plus once after the very last PV: completion
         // number t carries the scores of key tile t, and for the first tile of an item also "the previous item's O_x is
-        // complete" -- so the wait that ends an item is the wait that starts the next one.
-        int t = 0;  // key tiles processed so far (all items)
-        bool ok = true, waited = false;
+        // complete", which is what the write-out warps wait for.
+        int t = 0;       // key tiles processed so far (all items)
+        int n_done = 0;  // well-formed items finished so far
+        bool ok = true;
         auto item_done = [&]() {  // this warp is through with the item: its slot in the ring may be reused
             __syncwarp();
             if (lane == 0) {
@@ -612,24 +627,16 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         for (int k = 0; ok; ++k) {
             Item it;
             if (fetch_item<true>(sh, k, it, p.status, p.abort_word) <= 0) break;
-            if (it.malformed) {  // zero rows, latch
-                if (threadIdx.x == 128) atomicOr(p.status, EKV_DEV_FLAG_OOB);
-                if (row < it.rows_here) {
-                    uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)(it.qrow + row) * row_stride + (size_t)(it.head0 + x) * kD);
-#pragma unroll 1
-                    for (int c = 0; c < kD / 8; ++c) o[c] = make_uint4(0u, 0u, 0u, 0u);
-                }
+            if (it.malformed) {  // the write-out warps zero its rows
                 item_done();
                 continue;
             }
-            // only these four stay in registers over the key-tile loop; the write-out reads the rest from the ring again
             const int lim = it.prow + min(row, it.rows_here - 1);  // last key this row may see
             const int prow = it.prow, L = it.L, n_tiles = it.n_tiles;
             float m_run = -INFINITY, l_run = 0.f;
             for (int j = 0; j < n_tiles; ++j, ++t) {
                 const int s = t % kStages;
-                if (!waited) ok = wait_warp_inline(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
-                waited = false;
+                ok = wait_warp_inline(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
                 if (!ok) break;
                 fence_after();
                 const int key0 = j * kBN;
@@ -756,70 +763,118 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             }
             if (!ok) break;
 
-            // ---- write-out: O / l -> bf16 -> global.  The completion waited for here covers the item's last PV (and, if
-            // another item follows, its first QK^T: that wait is then not repeated).  The accumulator is read into
-            // registers in one go and handed back to the MMA warp at once; a thread holds a whole row, so the rows go
-            // through this warp's staging area (16-byte pieces XOR-swizzled by row) and leave as 128 contiguous bytes
-            // per row, four rows per instruction, one half of the channels at a time.
-            ok = wait_warp_inline(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
+            // ---- the rows' normalisers go to the write-out warps, and this warp is through with the item: the wait for the
+            // next item's first scores is the next thing it does
+            // (the write-out warps have read the previous item's normalisers once they have handed its O_x back: an item of
+            // one key tile can be through here before they have even started on the one before it)
+            if (n_done > 0) ok = wait_warp_inline(sh, O_FREE + x, (uint32_t)((n_done - 1) & 1), p.status, p.abort_word);
             if (!ok) break;
-            waited = true;
-            fence_after();
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            const int piece = lane & 7, sub = lane >> 3;
-            // A warp whose 32 rows all belong to the request hands each staged half to the TMA unit (one instruction, the
-            // rows leave asynchronously); a warp at the ragged end of a chunk writes its valid rows itself.
-            const uint4 slot0 = sh.item_slot(k)[0], slot2 = sh.item_slot(k)[2];  // the slot is this item's until item_done()
-            const int qrow = (int)slot0.y, rows_here = (int)slot0.w, head = (int)slot2.x + x;
-            const bool by_tma = wrow0 + 32 <= rows_here;
-            __nv_bfloat16 *dst = p.out + (size_t)qrow * row_stride + (size_t)head * kD + piece * 8;
-            // One half of the channels at a time, as a loop (not unrolled: this code runs once per item).  The accumulator
-            // is handed back after the second half has been read; nothing waits for it sooner, because the next item's
-            // first PV needs the P that these same warps produce after this write-out.
-#pragma unroll 1
-            for (int h2 = 0; h2 < 2; ++h2) {
-                float ov[64];
-                {
-                    uint32_t(&r)[64] = reinterpret_cast<uint32_t(&)[64]>(ov);
-                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[0]), t_o + 64 * h2);
-                    cp::tcgen05_ld_32x32b(reinterpret_cast<uint32_t(&)[32]>(r[32]), t_o + 64 * h2 + 32);
-                    cp::tcgen05_wait_ld();
-                }
-                uint4 v[8];
-#pragma unroll
-                for (int i = 0; i < 64; i += 8) {
-                    v[i >> 3].x = pack_bf16x2(ov[i] * inv, ov[i + 1] * inv);
-                    v[i >> 3].y = pack_bf16x2(ov[i + 2] * inv, ov[i + 3] * inv);
-                    v[i >> 3].z = pack_bf16x2(ov[i + 4] * inv, ov[i + 5] * inv);
-                    v[i >> 3].w = pack_bf16x2(ov[i + 6] * inv, ov[i + 7] * inv);
-                }
-                if (lane == 0) bulk_wait_group_read_0();  // the staging area is no longer being read by an earlier store
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    *reinterpret_cast<uint4 *>(stage + lane * 128 + ((i ^ (lane & 7)) << 4)) = v[i];  // = the 128-byte swizzle
-                if (by_tma) {
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_3d(&omap, smem_u32(stage), 64 * h2, head, qrow + wrow0);
-                        bulk_commit_group();
-                    }
-                } else {
-                    __syncwarp();
-#pragma unroll 1
-                    for (int r4 = 0; r4 < 8; ++r4) {
-                        const int lr = 4 * r4 + sub;  // row inside this warp's 32
-                        const uint4 w = *reinterpret_cast<const uint4 *>(stage + lr * 128 + ((piece ^ (lr & 7)) << 4));
-                        if (wrow0 + lr < rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)(wrow0 + lr) * row_stride + 64 * h2) = w;
-                    }
-                    __syncwarp();
-                }
-            }
-            fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(sh.bar(O_FREE + x));
+            sh.inv_l(x)[row] = l_run > 0.f ? 1.f / l_run : 0.f;
+            mbar_arrive(sh.bar(L_READY + x));
+            ++n_done;
             item_done();
+        }
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+        // =========================== write-out: O / l -> bf16 -> global ===========================
+        // Four warps, one per quarter of the TMEM lanes, take both heads of every item in turn.  With the write-out here
+        // the softmax warps go from an item's last tile straight to the next item's first, and their code is smaller by
+        // what this role holds (both matter for batches of short chunks, where an item is only a few key tiles long).
+        // The accumulator of a head is complete with the completion of S_READY that follows the item's last key tile; it is
+        // read 64 columns at a time and handed back to the MMA warp as soon as the second half is in registers.  A thread
+        // holds a whole row, so the rows go through a staging buffer (16-byte pieces XOR-swizzled by row) and leave as
+        // 128 contiguous bytes per row: a warp whose 32 rows all belong to the request hands each staged half to the
+        // TMA unit (one instruction, the rows leave asynchronously); a warp at the ragged end of a chunk writes its
+        // valid rows itself.  Each warp has two staging buffers and alternates between them.
+        const int wrow0 = (warp & 3) << 5;               // this warp's 32 rows of the tile = its TMEM lanes
+        const int row = wrow0 | lane;
+        const uint32_t lane_base = (uint32_t)wrow0 << 16;
+        uint8_t *stage0 = sh.ptr + kOffStage + (warp & 3) * 2 * kStageBytes;
+        const int piece = lane & 7, sub = lane >> 3;
+        int t = 0;       // key tiles of the well-formed items so far: completion number t of S_READY_x says O_x is complete
+        int n = 0;       // well-formed items so far
+        int buf = 0;     // staging buffer of the next half
+        int tma_buf = -1;  // buffer that the most recent store handed to the TMA unit reads from
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+            Item it;
+            if (fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;
+            if (it.malformed) {  // seq_len shorter than the chunk: zero rows, latch
+                if (threadIdx.x == 384) atomicOr(p.status, EKV_DEV_FLAG_OOB);
+                if (row < it.rows_here) {
+                    uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)(it.qrow + row) * row_stride + (size_t)it.head0 * kD);
+#pragma unroll 1
+                    for (int c = 0; c < 2 * kD / 8; ++c) o[c] = make_uint4(0u, 0u, 0u, 0u);  // both heads: adjacent in a row
+                }
+            } else {
+                t += it.n_tiles;
+                const bool by_tma = wrow0 + 32 <= it.rows_here;
+#pragma unroll 1
+                for (int x = 0; x < 2 && ok; ++x) {
+                    ok = wait_warp(sh, L_READY + x, (uint32_t)(n & 1), p.status, p.abort_word);
+                    if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
+                    if (!ok) break;
+                    fence_after();
+                    const float inv = sh.inv_l(x)[row];  // read before O_x is handed back: the softmax warps write the next item's late
+                    const uint32_t t_o = tmem + lane_base + col_o(x);
+                    __nv_bfloat16 *dst = p.out + (size_t)it.qrow * row_stride + (size_t)(it.head0 + x) * kD + piece * 8;
+#pragma unroll 1
+                    for (int h2 = 0; h2 < 2; ++h2) {
+                        // the buffer must no longer be read by an earlier store: the most recent one may still be if it
+                        // reads the other buffer
+                        if (lane == 0) {
+                            if (tma_buf == buf || !by_tma) bulk_wait_group_read_0();
+                            else bulk_wait_group_read_1();
+                        }
+                        __syncwarp();
+                        uint8_t *stage = stage0 + buf * kStageBytes;
+#pragma unroll 1
+                        for (int c2 = 0; c2 < 2; ++c2) {  // 32 columns at a time: this role lives on few registers
+                            float ov[32];
+                            tmem_ld32(ov, t_o + 64 * h2 + 32 * c2);
+                            if (h2 == 1 && c2 == 1) {  // all of O_x is in registers or staged: the next item's first PV may overwrite it
+                                fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(sh.bar(O_FREE + x));
+                            }
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                uint4 v;
+                                v.x = pack_bf16x2(ov[8 * i] * inv, ov[8 * i + 1] * inv);
+                                v.y = pack_bf16x2(ov[8 * i + 2] * inv, ov[8 * i + 3] * inv);
+                                v.z = pack_bf16x2(ov[8 * i + 4] * inv, ov[8 * i + 5] * inv);
+                                v.w = pack_bf16x2(ov[8 * i + 6] * inv, ov[8 * i + 7] * inv);
+                                *reinterpret_cast<uint4 *>(stage + lane * 128 + (((4 * c2 + i) ^ (lane & 7)) << 4)) = v;  // = the 128-byte swizzle
+                            }
+                        }
+                        if (by_tma) {
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                tma_store_3d(&omap, smem_u32(stage), 64 * h2, it.head0 + x, it.qrow + wrow0);
+                                bulk_commit_group();
+                            }
+                            tma_buf = buf;
+                        } else {
+                            __syncwarp();
+#pragma unroll 1
+                            for (int r4 = 0; r4 < 8; ++r4) {
+                                const int lr = 4 * r4 + sub;  // row inside this warp's 32
+                                const uint4 w = *reinterpret_cast<const uint4 *>(stage + lr * 128 + ((piece ^ (lr & 7)) << 4));
+                                if (wrow0 + lr < it.rows_here) *reinterpret_cast<uint4 *>(dst + (size_t)(wrow0 + lr) * row_stride + 64 * h2) = w;
+                            }
+                            __syncwarp();
+                        }
+                        buf ^= 1;
+                    }
+                }
+                ++n;
+            }
+            __syncwarp();  // this warp is through with the item: its slot in the ring may be reused
+            if (lane == 0) {
+                __threadfence_block();
+                atomicAdd(sh.done_count(), 1);
+            }
         }
         if (lane == 0) bulk_wait_group_0();  // every row this warp handed to the TMA unit has been written
     }

@@ -39,6 +39,11 @@ static constexpr int kSOffFlags = 8 * SNBAR;            // abort flag, TMEM base
 static constexpr int kSOffMask = kSOffFlags + 16;       // 2 slots x 4 masks
 static constexpr int kSOffItems = 320;                  // kSRing item slots of 64 bytes
 static_assert(kSOffMask + 32 <= kSOffItems, "barrier area");
+// This kernel's own thread count and register split (setmaxnreg: warps 0-3 drop to 72, warps 4-11 rise to 216; the raise
+// blocks until the registers are there, so the split has to fit the CTA's own allocation and the role code must match
+// the number of warps launched).
+static constexpr int kSThreads = 384, kSLaunchRegs = 168;
+static_assert(128 * 72 + 256 * 216 <= kSLaunchRegs * kSThreads && kSLaunchRegs * kSThreads <= 65536, "register split of the two-slot kernel");
 static constexpr int kSSmemBytes = kOffBar + kSOffItems + 64 * kSRing + 1024;  // + alignment slack
 static_assert(kSSmemBytes <= 232448, "shared memory of one CTA");
 
@@ -117,7 +122,7 @@ __device__ __forceinline__ int s_fetch_item(const SShared &sh, int k, Item &it, 
     return it.state == kItemWork ? 1 : 0;
 }
 
-__global__ void __launch_bounds__(kThreads, 1) prefill_tcs_kernel(const __grid_constant__ CUtensorMap kvmap,
+__global__ void __launch_bounds__(kSThreads, 1) prefill_tcs_kernel(const __grid_constant__ CUtensorMap kvmap,
                                                                   const __grid_constant__ CUtensorMap qmap,
                                                                   const __grid_constant__ CUtensorMap omap,
                                                                   const PrefillParams p) {
@@ -634,7 +639,7 @@ static ekv_status_t launch_prefill_tcs(ekv_pool *pool, int layer, const PrefillP
     const int grid = (int)(want < pool->sm_count ? want : pool->sm_count);
     cudaError_t e0 = cudaMemsetAsync(p.abort_word, 0, 2 * sizeof(int), stream);  // abort word + item counter
     if (e0 != cudaSuccess) return cuda_fail(e0, "ekv_attn_prefill_chunk: clear abort word and item counter");
-    prefill_tcs_kernel<<<grid, kThreads, kSSmemBytes, stream>>>(pool->kv_map[layer], qmap, omap, p);
+    prefill_tcs_kernel<<<grid, kSThreads, kSSmemBytes, stream>>>(pool->kv_map[layer], qmap, omap, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_prefill_chunk: launch");
     return EKV_OK;
