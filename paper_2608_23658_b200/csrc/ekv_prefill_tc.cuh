@@ -198,59 +198,38 @@ struct Shared {
 };
 
 // Bounded wait of a whole warp (every lane polls, all lanes agree on the outcome: the roles use warp-collective
-// instructions afterwards, so a warp must leave its loop as a whole).  It also gives up as soon as another role has
-// flagged an abort.  At the place that waits there is only one poll and a vote: a wait that is not over at once goes
-// on in ONE out-of-line copy of the polling loop.  (There are dozens of waits; with the loop, the clock and the
-// give-up path inlined at each, they were the largest part of the issuing warp's code, and the kernel has to stay
-// small enough for the instruction caches.)
-__device__ __noinline__ bool wait_slow(uint32_t b, uint32_t parity, volatile int *abort_flag, unsigned *status, int *abort_word) {
-    const uint64_t t0 = global_timer_ns();
-    bool ok = false;
-    for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(b, parity)) {
-            ok = true;
-            break;
-        }
-        if ((i & 31u) == 0u) {
-            if (*abort_flag) break;
-            if (global_timer_ns() - t0 > 2000000000ull) {
-                *abort_flag = 1;
-                *(volatile int *)abort_word = 1;
-                atomicOr(status, EKV_DEV_FLAG_TIMEOUT);
-                break;
-            }
-        }
-    }
-    return __all_sync(0xffffffffu, ok);
-}
-__device__ __forceinline__ bool wait_warp(const Shared &sh, int bar, uint32_t parity, unsigned *status, int *abort_word) {
-    const uint32_t b = sh.bar(bar);
-    if (__all_sync(0xffffffffu, mbar_try_wait(b, parity))) return true;
-    return wait_slow(b, parity, sh.abort_flag(), status, abort_word);
-}
-// The same with the loop inline, for the softmax warps: a call does not fit their register budget, and they wait in few places.
-__device__ __forceinline__ bool wait_warp_inline(const Shared &sh, int bar, uint32_t parity, unsigned *status, int *abort_word) {
-    const uint32_t b = sh.bar(bar);
-    bool ok = mbar_try_wait(b, parity);
-    if (!ok) {
-        const uint64_t t0 = global_timer_ns();
-        for (uint32_t i = 1;; ++i) {
-            if (mbar_try_wait(b, parity)) {
-                ok = true;
-                break;
-            }
-            if ((i & 31u) == 0u) {
-                if (*sh.abort_flag()) break;
-                if (global_timer_ns() - t0 > 2000000000ull) {
-                    *sh.abort_flag() = 1;
-                    *(volatile int *)abort_word = 1;
-                    atomicOr(status, EKV_DEV_FLAG_TIMEOUT);
-                    break;
-                }
-            }
-        }
-    }
-    return __all_sync(0xffffffffu, ok);
+// instructions afterwards, so a warp must leave its loop as a whole).  Nearly every wait is over within its first poll
+// (a poll sleeps in hardware until the phase completes or a time limit passes), so that case is one poll and a vote.
+// Otherwise the warp goes on polling in a loop of a dozen instructions, written in PTX so that it stays that small:
+// there are dozens of waits, and the kernel's code has to fit the instruction caches (with the loop, a clock and the
+// give-up path written out in C++ at each, the waits were the largest part of the issuing warp's code; as a call to one
+// out-of-line copy they cost register spills around every call).  The loop gives up as soon as another role of the CTA
+// has given up.  Its bound is a number of polls: a failed mbarrier.try_wait sleeps about 1.5 us on this part (measured:
+// 2900 cycles a poll, whatever the number of polling warps), so kPollLimit polls are about three seconds.  A wait that
+// runs out leaves 2 in the CTA's abort flag; the teardown turns that into EKV_ERR_TIMEOUT.
+static constexpr uint32_t kPollLimit = 1u << 21;
+__device__ __forceinline__ bool wait_warp(const Shared &sh, int bar, uint32_t parity) {
+    if (__all_sync(0xffffffffu, mbar_try_wait(sh.bar(bar), parity))) return true;  // the usual case: over within the first poll
+    uint32_t ok;
+    // poll; done if the phase is over; give up if the CTA's abort flag is up; count; after kPollLimit polls raise the flag (2)
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 i, f;\n\tmov.u32 i, 0;\n"
+        "WAIT_POLL:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra WAIT_OUT;\n\t"
+        "ld.volatile.shared.u32 f, [%3];\n\t"
+        "setp.ne.u32 q, f, 0;\n\t"
+        "@q bra WAIT_OUT;\n\t"
+        "add.u32 i, i, 1;\n\t"
+        "setp.lt.u32 q, i, %4;\n\t"
+        "@q bra WAIT_POLL;\n\t"
+        "st.volatile.shared.u32 [%3], 2;\n"
+        "WAIT_OUT:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(sh.bar(bar)), "r"(parity), "r"(sh.base + kOffBar + 8 * NBAR), "n"(kPollLimit)
+        : "memory");
+    return __all_sync(0xffffffffu, ok != 0u);
 }
 
 // One work item.  The scheduler decodes it (that takes dependent reads of device memory) and posts it in the ring;
@@ -303,10 +282,8 @@ __device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item 
 
 // The CTA's k-th item as posted by the scheduler.  Returns 1 for an item to work on, 0 at the end of the list (or for
 // an item that names no request), -1 if the wait was given up.  A malformed item still counts as 1.
-template <bool kInlineWait = false>
-__device__ __forceinline__ int fetch_item(const Shared &sh, int k, Item &it, unsigned *status, int *abort_word) {
-    const bool got = kInlineWait ? wait_warp_inline(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1), status, abort_word)
-                                 : wait_warp(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1), status, abort_word);
+__device__ __forceinline__ int fetch_item(const Shared &sh, int k, Item &it) {
+    const bool got = wait_warp(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1));
     if (!got) return -1;
     const uint4 *src = sh.item_slot(k);
     const uint4 a = src[0], b = src[1], c = src[2];  // field by field: the struct stays in registers
@@ -385,7 +362,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         bool ok = true;
         for (int k = 0; ok; ++k) {
             Item it;
-            if (fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;
+            if (fetch_item(sh, k, it) <= 0) break;
             if (it.malformed) continue;
             const int *bt = p.block_tables + (size_t)it.req * p.max_blocks;
             auto load_id = [&](int j) {  // lane l: id of block 8j + l%8 (-1 past the end, -2 invalid)
@@ -410,7 +387,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 const int b = lane & 15, blk = b >> 1, half = b & 1;
                 const int my_id = __shfl_sync(0xffffffffu, id, blk);
                 const int row = it.g * 16 + kv_row_off;  // row inside the block: (K|V, kv-head, token)
-                if (t >= kStages && !wait_warp(sh, EMPTY + s, (uint32_t)(((t / kStages) - 1) & 1), p.status, p.abort_word)) {
+                if (t >= kStages && !wait_warp(sh, EMPTY + s, (uint32_t)(((t / kStages) - 1) & 1))) {
                     ok = false;
                     break;
                 }
@@ -447,9 +424,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                         if (!got && (i & 31u) == 31u) {
                             if (*sh.abort_flag()) return false;
                             if (global_timer_ns() - t0 > 2000000000ull) {
-                                *sh.abort_flag() = 1;
-                                *(volatile int *)p.abort_word = 1;
-                                atomicOr(p.status, EKV_DEV_FLAG_TIMEOUT);
+                                *sh.abort_flag() = 2;
                                 return false;
                             }
                         }
@@ -478,12 +453,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             ok = post_until(k + kItemAhead);
             if (!ok || k >= posted) break;
             Item it;
-            if (fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;  // posted by this warp: the wait passes at once
+            if (fetch_item(sh, k, it) <= 0) break;  // posted by this warp: the wait passes at once
             if (it.malformed) continue;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 // the previous item's last QK^T of this head has read the tile
-                if (n > 0 && !wait_warp(sh, Q_EMPTY + x, (uint32_t)((n - 1) & 1), p.status, p.abort_word)) {
+                if (n > 0 && !wait_warp(sh, Q_EMPTY + x, (uint32_t)((n - 1) & 1))) {
                     ok = false;
                     break;
                 }
@@ -542,7 +517,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             have_nxt = false;  // next well-formed item of this CTA, if any
             while (list_ok && !list_end && !have_nxt) {
                 Item it;
-                const int st = fetch_item(sh, k_item++, it, p.status, p.abort_word);
+                const int st = fetch_item(sh, k_item++, it);
                 if (st < 0) list_ok = false;
                 else if (st == 0) list_end = true;
                 else have_nxt = !it.malformed;
@@ -560,17 +535,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 const int s1 = t % kStages;                       // its stage
                 // that tile is the last one of its item: its QK^T is the last reader of the item's Q tile
                 const bool next_closes = new_item ? nxt_tiles == 1 : j + 2 == cur_tiles;
-                if (pv) ok = wait_warp(sh, V_FULL + s, (uint32_t)((tv / kStages) & 1), p.status, p.abort_word);
+                if (pv) ok = wait_warp(sh, V_FULL + s, (uint32_t)((tv / kStages) & 1));
 #pragma unroll
                 for (int x = 0; x < 2 && ok; ++x) {
                     if (pv) {
                         // O_x still holds the previous item's result until its write-out has read it
-                        if (j == 0 && n_now > 1) ok = wait_warp(sh, O_FREE + x, (uint32_t)((n_now - 2) & 1), p.status, p.abort_word);
-                        if (ok) ok = wait_warp(sh, P_PART + x, (uint32_t)(tv & 1), p.status, p.abort_word);
+                        if (j == 0 && n_now > 1) ok = wait_warp(sh, O_FREE + x, (uint32_t)((n_now - 2) & 1));
+                        if (ok) ok = wait_warp(sh, P_PART + x, (uint32_t)(tv & 1));
                         if (!ok) break;
                         fence_after();
                         issue_pv(x, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
-                        ok = wait_warp(sh, P_READY + x, (uint32_t)(tv & 1), p.status, p.abort_word);
+                        ok = wait_warp(sh, P_READY + x, (uint32_t)(tv & 1));
                         if (!ok) break;
                         fence_after();
                         issue_pv(x, s, true, kPartSteps, kBN / 16);
@@ -578,8 +553,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                     }
                     if (more) {
                         // a new item: its Q tile of head x must have landed; head A also checks the K tile
-                        if (new_item) ok = wait_warp(sh, Q_FULL + x, (uint32_t)(n_now & 1), p.status, p.abort_word);
-                        if (ok && x == 0) ok = wait_warp(sh, K_FULL + s1, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
+                        if (new_item) ok = wait_warp(sh, Q_FULL + x, (uint32_t)(n_now & 1));
+                        if (ok && x == 0) ok = wait_warp(sh, K_FULL + s1, (uint32_t)((t / kStages) & 1));
                         if (!ok) break;
                         fence_after();
                         issue_qk(x, s1);
@@ -599,7 +574,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         }
         // every MMA this thread issued must be finished before TMEM is released
         mma_commit(sh.bar(DRAIN));
-        (void)wait_warp(sh, DRAIN, 0, p.status, p.abort_word);
+        (void)wait_warp(sh, DRAIN, 0);
     }
     } else if (warp < 12) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 184;");
@@ -626,7 +601,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         };
         for (int k = 0; ok; ++k) {
             Item it;
-            if (fetch_item<true>(sh, k, it, p.status, p.abort_word) <= 0) break;
+            if (fetch_item(sh, k, it) <= 0) break;
             if (it.malformed) {  // the write-out warps zero its rows
                 item_done();
                 continue;
@@ -636,7 +611,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             float m_run = -INFINITY, l_run = 0.f;
             for (int j = 0; j < n_tiles; ++j, ++t) {
                 const int s = t % kStages;
-                ok = wait_warp_inline(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
+                ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1));
                 if (!ok) break;
                 fence_after();
                 const int key0 = j * kBN;
@@ -646,7 +621,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 // (unwritten slots): their V rows must not reach the tensor pipe, because 0 * NaN = NaN
                 const bool dirty_v = (key0 + kBN > L) || bad != 0;
                 if (dirty_v && x == 0) {
-                    ok = wait_warp_inline(sh, V_FULL + s, (uint32_t)((t / kStages) & 1), p.status, p.abort_word);
+                    ok = wait_warp(sh, V_FULL + s, (uint32_t)((t / kStages) & 1));
                     if (!ok) break;
                     uint8_t *vdst = sh.ptr + kOffV + s * kTileBytes;
                     if ((key0 + row >= L) || ((bad >> (row >> 4)) & 1)) {  // thread `row` owns key row `row` of the tile
@@ -767,7 +742,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             // next item's first scores is the next thing it does
             // (the write-out warps have read the previous item's normalisers once they have handed its O_x back: an item of
             // one key tile can be through here before they have even started on the one before it)
-            if (n_done > 0) ok = wait_warp_inline(sh, O_FREE + x, (uint32_t)((n_done - 1) & 1), p.status, p.abort_word);
+            if (n_done > 0) ok = wait_warp(sh, O_FREE + x, (uint32_t)((n_done - 1) & 1));
             if (!ok) break;
             sh.inv_l(x)[row] = l_run > 0.f ? 1.f / l_run : 0.f;
             mbar_arrive(sh.bar(L_READY + x));
@@ -798,7 +773,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         bool ok = true;
         for (int k = 0; ok; ++k) {
             Item it;
-            if (fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;
+            if (fetch_item(sh, k, it) <= 0) break;
             if (it.malformed) {  // seq_len shorter than the chunk: zero rows, latch
                 if (threadIdx.x == 384) atomicOr(p.status, EKV_DEV_FLAG_OOB);
                 if (row < it.rows_here) {
@@ -811,8 +786,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 const bool by_tma = wrow0 + 32 <= it.rows_here;
 #pragma unroll 1
                 for (int x = 0; x < 2 && ok; ++x) {
-                    ok = wait_warp(sh, L_READY + x, (uint32_t)(n & 1), p.status, p.abort_word);
-                    if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1), p.status, p.abort_word);
+                    ok = wait_warp(sh, L_READY + x, (uint32_t)(n & 1));
+                    if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1));
                     if (!ok) break;
                     fence_after();
                     const float inv = sh.inv_l(x)[row];  // read before O_x is handed back: the softmax warps write the next item's late
@@ -884,6 +859,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     __syncthreads();
     fence_after();
     if (*sh.abort_flag()) {
+        if (threadIdx.x == 0) {  // a wait of this CTA ran out: latch it, and tell the launch's other CTAs
+            *(volatile int *)p.abort_word = 1;
+            atomicOr(p.status, EKV_DEV_FLAG_TIMEOUT);
+        }
         if (warp == 0 || warp == 2) {
             const int FULL = warp == 2 ? V_FULL : K_FULL;
             for (int j = max(0, tiles_issued - kStages); j < tiles_issued; ++j)
