@@ -159,6 +159,10 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
         "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar)
         : "memory");
 }
+// the same from inside a branch that one elected lane has taken
+__device__ __forceinline__ void mma_commit_one(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -476,19 +480,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         // descriptor low words of the tile origins; stepping inside a tile adds a compile-time constant
         const uint32_t q_lo0 = desc_lo(sh.base + kOffQ, 16);
         const uint32_t k_lo0 = desc_lo(sh.base + kOffK, 16), v_lo0 = desc_lo(sh.base + kOffV, kHalfBytes);
-        auto issue_qk = [&](int x, int s) {  // S_x = Q_x K(s)^T
-            if (elect_one()) {
-                const uint64_t hi = (uint64_t)kDescHi << 32;
-                const uint64_t k_desc = hi | (k_lo0 + (uint32_t)s * (kTileBytes >> 4)), q_desc = hi | (q_lo0 + (uint32_t)x * (kTileBytes >> 4));
-                const uint32_t d = tmem + col_s(x);
-#pragma unroll
-                for (int k = 0; k < kD / 16; ++k) {
-                    const uint32_t off = ((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4;
-                    mma_ss(d, q_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
-                }
-            }
-            __syncwarp();
-        };
         auto issue_pv = [&](int x, int s, bool acc, int k0, int k1) {  // O_x (+)= P_x[:, 16k0:16k1] V(s)[16k0:16k1, :]
             if (elect_one()) {
                 const uint64_t v_desc = ((uint64_t)kDescHi << 32) | (v_lo0 + (uint32_t)s * (kTileBytes >> 4));
@@ -547,21 +538,40 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                         issue_pv(x, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
                         ok = wait_warp(sh, P_READY + x, (uint32_t)(tv & 1));
                         if (!ok) break;
-                        fence_after();
-                        issue_pv(x, s, true, kPartSteps, kBN / 16);
-                        if (x == 1) mma_commit(sh.bar(V_EMPTY + s));
                     }
                     if (more) {
                         // a new item: its Q tile of head x must have landed; head A also checks the K tile
                         if (new_item) ok = wait_warp(sh, Q_FULL + x, (uint32_t)(n_now & 1));
                         if (ok && x == 0) ok = wait_warp(sh, K_FULL + s1, (uint32_t)((t / kStages) & 1));
                         if (!ok) break;
-                        fence_after();
-                        issue_qk(x, s1);
-                        if (next_closes) mma_commit(sh.bar(Q_EMPTY + x));
-                        if (x == 1) mma_commit(sh.bar(K_EMPTY + s1));
                     }
-                    mma_commit(sh.bar(S_READY + x));  // scores of the next tile, and (after an item's last tile) O_x complete
+                    fence_after();
+                    // The rest of the step in one go, by one elected lane: the last quarter of PV, QK^T of the next tile, and
+                    // the commits (this is the stretch between "P is there" and "the next scores are there" on every
+                    // head's critical chain, so it is as few instructions as it can be).
+                    if (elect_one()) {
+                        const uint64_t hi = (uint64_t)kDescHi << 32;
+                        if (pv) {
+                            const uint64_t v_desc = hi | (v_lo0 + (uint32_t)s * (kTileBytes >> 4));
+                            const uint32_t d = tmem + col_o(x), a = tmem + col_s(x);
+#pragma unroll
+                            for (int k = kPartSteps; k < kBN / 16; ++k) mma_ts(d, a + 8 * k, v_desc + ((k * 2048) >> 4), kIdescPV, 1u);
+                            if (x == 1) mma_commit_one(sh.bar(V_EMPTY + s));
+                        }
+                        if (more) {
+                            const uint64_t k_desc = hi | (k_lo0 + (uint32_t)s1 * (kTileBytes >> 4)), q_desc = hi | (q_lo0 + (uint32_t)x * (kTileBytes >> 4));
+                            const uint32_t d = tmem + col_s(x);
+#pragma unroll
+                            for (int k = 0; k < kD / 16; ++k) {
+                                const uint32_t off = ((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4;
+                                mma_ss(d, q_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
+                            }
+                            if (next_closes) mma_commit_one(sh.bar(Q_EMPTY + x));
+                            if (x == 1) mma_commit_one(sh.bar(K_EMPTY + s1));
+                        }
+                        mma_commit_one(sh.bar(S_READY + x));  // scores of the next tile, and (after an item's last tile) O_x complete
+                    }
+                    __syncwarp();
                 }
                 if (!ok) break;
                 if (pv) ++tv;
