@@ -573,6 +573,33 @@ def test_prefill_edge_cases_bad_ids_empty_requests_negative_scale(prefill_kernel
         pool.close()
 
 
+def test_prefill_request_with_fewer_keys_than_rows_is_zeroed_and_latched(prefill_kernel):
+    """A request whose seq_len is smaller than its chunk (no valid prefix) is invalid: its rows come out as zeros,
+    EKV_ERR_BLOCK_OOB is latched, and the requests around it are served as usual (every prefill kernel)."""
+    shape = I.LLAMA8B
+    chunks = [(20, 140), (0, 200), (300, 129)]                    # (prefix, rows)
+    lengths = [p + c for p, c in chunks]
+    case = Case(shape, lengths, int(I.blocks_for(torch.tensor(lengths), 16).sum()) + 9, 101)
+    try:
+        cu = torch.tensor(np.cumsum([0] + [c for _, c in chunks]), dtype=torch.int32)
+        q = rand_q(102, int(cu[-1]), shape)
+        scale = 1 / math.sqrt(shape.head_dim)
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q, case.tables,
+                                         cu, case.lengths, scale)
+        short = case.d_lengths.clone()
+        short[1] = 150                                             # 200 rows over 150 keys
+        out = torch.full((int(cu[-1]), shape.num_q_heads, shape.head_dim), 7.0, dtype=torch.bfloat16, device=DEV)
+        case.pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, short, scale, out=out)
+        torch.cuda.synchronize()
+        assert case.pool.poll_status() == ekv.Status.ERR_BLOCK_OOB
+        a, b = int(cu[1]), int(cu[2])
+        assert torch.equal(out[a:b], torch.zeros_like(out[a:b]))
+        check_close(out[:a], want[:a], "request before the invalid one")
+        check_close(out[b:], want[b:], "request after the invalid one")
+    finally:
+        case.close()
+
+
 def test_prefill_calls_in_flight_on_two_streams_keep_their_own_work_lists():
     """Two chunked-prefill calls of one pool running at the same time (two streams, different requests): the persistent
     kernel hands out its work items from a counter in device memory, and every launch must have its own."""
