@@ -27,8 +27,8 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
     }
     // Kernels (scale > 0 unless stated):
     //   two-head tcgen05 kernel   head_dim 128, even query group: a persistent CTA per SM, every K/V tile feeds two heads.
-    //                             Measured, 32768 query tokens in one call: 256 x 128 fresh prompts 134 us against 161 us
-    //                             for the two-slot kernel; 64 x 512: 236 against 335; 16 x 2048: 545 against 770
+    //                             Measured, 32768 query tokens in one call: 256 x 128 fresh prompts 130 us against 161 us
+    //                             for the two-slot kernel; 64 x 512: 198 against 335-364; 16 x 2048: 508 against 769
     //   two-slot tcgen05 kernel   head_dim 128, one head per work item, the CTA's two TMEM slots on their own clocks: odd
     //                             query groups
     //   one-head tcgen05 kernel   head_dim 64 (one CTA per tile and head, two CTAs per SM)

@@ -81,6 +81,7 @@ static constexpr float kRescaleThreshold = 8.f;        // log2 units
 static constexpr int kLaunchRegs = 128, kRegsUtil = 72, kRegsSoftmax = 184, kRegsOut = 72;
 static_assert(128 * (kRegsUtil + kRegsOut) + 256 * kRegsSoftmax <= kLaunchRegs * kThreads, "setmaxnreg split exceeds the CTA's registers");
 static_assert(kLaunchRegs * kThreads <= 65536 && kRegsUtil % 8 == 0 && kRegsSoftmax % 8 == 0 && kRegsOut % 8 == 0, "register split");
+static_assert(kRegsUtil == 72 && kRegsSoftmax == 184 && kRegsOut == 72, "the setmaxnreg instructions in the kernel carry these numbers as literals");
 
 // shared-memory map (offsets from the 1024-byte aligned base)
 static constexpr int kOffQ = 0;                                   // Q_A, Q_B

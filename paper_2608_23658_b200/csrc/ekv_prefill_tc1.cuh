@@ -39,6 +39,7 @@ static constexpr uint32_t kColS = 0, kColO = 128;
 static constexpr int kLaunchRegs = 128, kRegsUtil = 40, kRegsSoftmax = 216;
 static_assert(128 * kRegsUtil + 128 * kRegsSoftmax <= kLaunchRegs * kThreads, "setmaxnreg split exceeds the CTA's registers");
 static_assert(2 * kLaunchRegs * kThreads <= 65536 && kRegsUtil % 8 == 0 && kRegsSoftmax % 8 == 0, "two CTAs per SM");
+static_assert(kRegsUtil == 40 && kRegsSoftmax == 216 && kThreads == 256, "the setmaxnreg instructions and the role split in the kernel carry these numbers as literals");
 
 template <int D>
 struct Geo {
