@@ -403,8 +403,9 @@ EKV_API ekv_status_t ekv_controller_stats(const ekv_controller_t *ctrl, ekv_cont
  * ekv_selftest_bounded_wait -- ours (error handling; the paper has no counterpart).  Every wait inside
  * the kernels is bounded: when it runs out, the kernel latches EKV_ERR_TIMEOUT, finishes, and the
  * context stays usable.  This call runs that path on purpose and harmlessly: it enqueues on `stream`
- * one small kernel that waits, with the kernels' own wait routine and a limit of limit_us microseconds
- * (1 .. 100000), on a barrier that nothing arrives on.  After the stream has been synchronised
+ * one small kernel that waits, with the kernels' own wait routines (the one bounded by a clock, then the
+ * one bounded by a number of polls) and a limit of limit_us microseconds each (1 .. 100000), on a barrier
+ * that nothing arrives on.  After the stream has been synchronised
  * ekv_poll_status returns EKV_ERR_TIMEOUT once, and every other call keeps working.
  * waited_ns_device: DEVICE uint64, or NULL; receives how long the wait lasted.
  */

@@ -215,26 +215,7 @@ struct Shared {
 static constexpr uint32_t kPollLimit = 1u << 21;
 __device__ __forceinline__ bool wait_warp(const Shared &sh, int bar, uint32_t parity) {
     if (__all_sync(0xffffffffu, mbar_try_wait(sh.bar(bar), parity))) return true;  // the usual case: over within the first poll
-    uint32_t ok;
-    // poll; done if the phase is over; give up if the CTA's abort flag is up; count; after kPollLimit polls raise the flag (2)
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .u32 i, f;\n\tmov.u32 i, 0;\n"
-        "WAIT_POLL:\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "@p bra WAIT_OUT;\n\t"
-        "ld.volatile.shared.u32 f, [%3];\n\t"
-        "setp.ne.u32 q, f, 0;\n\t"
-        "@q bra WAIT_OUT;\n\t"
-        "add.u32 i, i, 1;\n\t"
-        "setp.lt.u32 q, i, %4;\n\t"
-        "@q bra WAIT_POLL;\n\t"
-        "st.volatile.shared.u32 [%3], 2;\n"
-        "WAIT_OUT:\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(sh.bar(bar)), "r"(parity), "r"(sh.base + kOffBar + 8 * NBAR), "n"(kPollLimit)
-        : "memory");
-    return __all_sync(0xffffffffu, ok != 0u);
+    return __all_sync(0xffffffffu, mbar_wait_polls(sh.bar(bar), parity, sh.base + kOffBar + 8 * NBAR, kPollLimit));
 }
 
 // One work item.  The scheduler decodes it (that takes dependent reads of device memory) and posts it in the ring;

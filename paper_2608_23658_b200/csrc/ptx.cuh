@@ -65,6 +65,32 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_
     }
 }
 
+// The same wait bounded by a number of polls instead of a clock, as a loop of a dozen instructions: poll; done if the
+// phase is over; give up if the word at abort_flag (shared-window address) is not zero; count; after max_polls failed polls
+// store 2 there and give up.  A failed try_wait sleeps in hardware (about 1.5 us on B200, measured), so the bound is a time
+// bound all the same.  Returns false if it gave up.
+__device__ __forceinline__ bool mbar_wait_polls(uint32_t bar, uint32_t parity, uint32_t abort_flag, uint32_t max_polls) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 i, f;\n\tmov.u32 i, 0;\n"
+        "WAIT_POLL:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra WAIT_OUT;\n\t"
+        "ld.volatile.shared.u32 f, [%3];\n\t"
+        "setp.ne.u32 q, f, 0;\n\t"
+        "@q bra WAIT_OUT;\n\t"
+        "add.u32 i, i, 1;\n\t"
+        "setp.lt.u32 q, i, %4;\n\t"
+        "@q bra WAIT_POLL;\n\t"
+        "st.volatile.shared.u32 [%3], 2;\n"
+        "WAIT_OUT:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(abort_flag), "r"(max_polls)
+        : "memory");
+    return ok != 0u;
+}
+
 // ---- TMA: tiled loads global -> shared, completion on an mbarrier of the issuing CTA --------------
 // 3-D tiled loads: coordinates (channel, row inside the block, block id)
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, int x, int y, int z, uint32_t bar) {
