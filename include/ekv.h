@@ -84,12 +84,12 @@ enum {
                                     instead of one range and two handles per layer (see above) */
     EKV_PREFILL_ONE_HEAD = 1u << 4, /* ekv_pool_create: ekv_attn_prefill_chunk on this pool always runs a
                                     tcgen05 kernel whose work item is ONE query head (normally chosen for
-                                    head_dim 64 and odd query groups), so that it can be tested and timed
-                                    on any shape. */
+                                    head_dim 64 and for query groups of one), so that it can be tested and
+                                    timed on any shape. */
     EKV_PREFILL_TWO_HEAD = 1u << 5, /* ekv_pool_create: ekv_attn_prefill_chunk on this pool runs the two-head
-                                    tcgen05 kernel whenever the shape allows it (head_dim 128, even query
-                                    group, scale > 0).  That is also the default choice for such a shape;
-                                    the flag states it. */
+                                    tcgen05 kernel whenever the shape allows it (head_dim 128, query groups
+                                    of two or more heads, scale > 0).  That is also the default choice for
+                                    such a shape; the flag states it. */
     EKV_PREFILL_WARP_MMA = 1u << 3 /* ekv_pool_create: ekv_attn_prefill_chunk on this pool always runs the
                                     warp-level (mma.sync) kernel, never a tcgen05 one.  Same results within
                                     the stated tolerance; exists so the two kernel families can be checked

@@ -26,22 +26,25 @@ extern "C" ekv_status_t ekv_attn_prefill_chunk(ekv_pool_t *pool, int32_t layer, 
         return EKV_ERR_INVALID;
     }
     // Kernels (scale > 0 unless stated):
-    //   two-head tcgen05 kernel   head_dim 128, even query group: a persistent CTA per SM, every K/V tile feeds two heads.
-    //                             Measured, 32768 query tokens in one call: 256 x 128 fresh prompts 130 us against 161 us
-    //                             for the two-slot kernel; 64 x 512: 198 against 335-364; 16 x 2048: 508 against 769
-    //   two-slot tcgen05 kernel   head_dim 128, one head per work item, the CTA's two TMEM slots on their own clocks: odd
-    //                             query groups
+    //   two-head tcgen05 kernel   head_dim 128, query groups of 2 or more: a persistent CTA per SM, every K/V tile feeds two
+    //                             heads (an odd group is cut into pairs and one single-head item per kv-head).
+    //                             Measured, 32768 query tokens in one call, 32q/8kv: 256 x 128 fresh prompts 130 us against
+    //                             161 us for the two-slot kernel; 64 x 512: 198 against 335-364; 16 x 2048: 508 against
+    //                             769.  28q/4kv (groups of 7): a 16384-token prompt 1.63 against 2.11 ms, 64 x 512 215
+    //                             against 299 us
+    //   two-slot tcgen05 kernel   head_dim 128, one head per work item, the CTA's two TMEM slots on their own clocks: query
+    //                             groups of one (no two heads share a K/V tile)
     //   one-head tcgen05 kernel   head_dim 64 (one CTA per tile and head, two CTAs per SM)
     //   warp-level MMA kernel     non-positive scales, and every call on a pool created with EKV_PREFILL_WARP_MMA (which
     //                             the tests use to check the kernel families against each other)
-    // EKV_PREFILL_ONE_HEAD forces the one-head family on an even group; EKV_PREFILL_TWO_HEAD is what an even group at
+    // EKV_PREFILL_ONE_HEAD forces the one-head family on any group; EKV_PREFILL_TWO_HEAD is what a group of two or more at
     // head_dim 128 gets anyway (kept so that a caller can say so).
     const int group = pool->desc.num_q_heads / pool->desc.num_kv_heads;
     const uint32_t pf = pool->desc.flags;
     enum { K_TWO_HEAD, K_ONE_HEAD, K_WARP_MMA } kernel;
     if ((pf & EKV_PREFILL_WARP_MMA) || !(scale > 0.f)) {
         kernel = K_WARP_MMA;
-    } else if ((pf & EKV_PREFILL_ONE_HEAD) || pool->desc.head_dim != 128 || group % 2 != 0) {
+    } else if ((pf & EKV_PREFILL_ONE_HEAD) || pool->desc.head_dim != 128 || group == 1) {
         kernel = K_ONE_HEAD;
     } else {
         kernel = K_TWO_HEAD;

@@ -1,9 +1,14 @@
 // Chunked-prefill attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM),
-// head_dim 128, even query group.  PERSISTENT: one CTA per SM walks a list of work items.
+// head_dim 128, query groups of two or more heads.  PERSISTENT: one CTA per SM walks a list of work
+// items.
 //
 // Work item = 128 query positions of one request x TWO query heads (A, B) that share a kv-head, so
 // every K/V tile staged in shared memory feeds two 128x128 score tiles (ping-pong: while the
-// softmax warps work on one head's scores the tensor pipe runs the other head's MMAs).  Items are
+// softmax warps work on one head's scores the tensor pipe runs the other head's MMAs).  A kv group
+// with an odd number of query heads (7 for a 28 / 4 model) is cut into pairs and ONE item of a single
+// head, which head B's warps sit out; the barriers of a head then count that head's own tiles and
+// items, and where a head's last PV and its next first QK^T are no longer one commit the roles take
+// care not to wait on a phase parity from two completions away (notes at those places).  Items are
 // ordered head pair by head pair and, inside a pair, from the heaviest (latest) query tile to the
 // lightest, and are handed out dynamically: warp 3 draws item numbers from a counter in device
 // memory and posts them in a small ring in shared memory, from which every role of the CTA reads
@@ -91,7 +96,7 @@ static constexpr int kOffStage = kOffV + kStages * kTileBytes;    // write-out s
 static constexpr int kStageBytes = 32 * 128;
 static constexpr int kOffBar = kOffStage + 8 * kStageBytes;       // mbarriers
 static constexpr int kOffInvL = kOffBar + 512;                     // 1 / row sum of the finished item: [2 heads][128 rows] floats
-static constexpr int kSmemBytes = kOffInvL + 1024 + 1024;         // barriers, flags, item ring; row sums; + alignment slack
+static constexpr int kSmemBytes = kOffInvL + 1024 + 64 + 1024;         // barriers, flags, item ring; row sums; + alignment slack
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
 // barrier slots (8 bytes each)
@@ -193,10 +198,12 @@ struct Shared {
     // key-tile count: the K producer may run two tiles ahead of the softmax warps (it only waits for the QK MMAs), so a
     // slot per STAGE would be overwritten before the softmax of the older tile has read it.
     __device__ __forceinline__ volatile int *bad_mask(int tile) const { return (volatile int *)(ptr + kOffBar + 8 * NBAR + 16 + 4 * (tile & 3)); }
-    // Softmax and write-out warps that are through with an item (12 per item) are COUNTED, not signalled on an mbarrier: the scheduler
-    // looks at the count only when it needs a ring slot back, possibly a few items later, and a phase parity cannot tell
-    // "not yet" from "two phases ago".
-    __device__ __forceinline__ int *done_count() const { return (int *)(ptr + kOffBar + 8 * NBAR + 12); }
+    // Every softmax and write-out warp (12 of them) keeps, in a word of its own, the number of items it is through with, and
+    // the scheduler gives a ring slot to a new item once ALL twelve are past the old one.  Not an mbarrier: the scheduler
+    // looks only when it needs a slot back, possibly a few items later, and a phase parity cannot tell "not yet" from "two
+    // phases ago".  Not one shared count either: the warps of head B skip the items that have one head, and a sum would
+    // let their lead pay for a warp that lags.
+    __device__ __forceinline__ volatile int *items_done(int w12) const { return (volatile int *)(ptr + kOffInvL + 1024) + w12; }
     __device__ __forceinline__ float *inv_l(int x) const { return (float *)(ptr + kOffInvL) + 128 * x; }
     // items posted by the scheduler: slot k % kItemRing holds the CTA's k-th item
     __device__ __forceinline__ uint4 *item_slot(int k) const { return (uint4 *)(ptr + kOffBar + 256 + 64 * (k % kItemRing)); }
@@ -227,7 +234,7 @@ struct Item {
     int rows_here;  // rows of the tile that belong to the request (1..128)
     int L, n_tiles, n_blocks;  // keys of the request; key tiles / blocks any row of this tile may see
     int head0, g;   // first of the two query heads; their kv-head
-    int spare;
+    int nh;         // query heads of the item: 2, or 1 for the odd head of a kv group with an odd number of query heads
     int malformed;  // seq_len shorter than the chunk: rows are zero-filled, nothing is loaded or multiplied
     int state;      // kItemWork, or kItemEnd: the list of this CTA ends here
 };
@@ -238,9 +245,10 @@ static_assert(sizeof(Item) == 48, "item slot");
 // tile.  One group per launch makes the list globally longest-first (the end of the launch is made of one-tile items,
 // so the CTAs finish together); smaller groups keep fewer kv-heads' K/V streaming through L2 at a time.
 static constexpr int kPairGroup = EKV_TC_PAIR_GROUP;
+__host__ __device__ __forceinline__ int head_pairs(const PrefillParams &p) { return p.num_kv_heads * ((p.group + 1) / 2); }
 __device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item &it) {
     it.state = kItemWork;
-    const int npairs = p.num_q_heads / 2;
+    const int npairs = head_pairs(p);
     const int gp = kPairGroup > 0 ? kPairGroup : npairs;
     const int per_group = p.q_tiles * gp;
     const int grp = m / per_group, r = m - grp * per_group;
@@ -250,8 +258,10 @@ __device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item 
     const int tile_idx = p.q_tiles - 1 - rank;              // heaviest (latest) tiles first
     int acc_tiles = 0, c_r = 0, q0 = 0;
     if (!find_request(p, tile_idx, kBM, it.req, acc_tiles, q0, c_r)) return false;
-    it.head0 = 2 * pair;
-    it.g = it.head0 / p.group;
+    const int per_kv = (p.group + 1) / 2;  // a kv group of g query heads is g / 2 pairs, plus a single head if g is odd
+    it.g = pair / per_kv;
+    it.head0 = it.g * p.group + 2 * (pair - it.g * per_kv);
+    it.nh = min(2, (it.g + 1) * p.group - it.head0);
     const int row0 = (tile_idx - acc_tiles) * kBM;
     it.L = min(p.seq_lens[it.req], p.max_blocks * 16);
     const int prefix = it.L - c_r;
@@ -259,7 +269,6 @@ __device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item 
     it.prow = prefix + row0;
     it.rows_here = min(kBM, c_r - row0);
     it.malformed = prefix < 0 ? 1 : 0;
-    it.spare = 0;
     const int kv_end = min(it.L, it.prow + it.rows_here);  // keys any row of this tile may see
     it.n_tiles = (kv_end + kBN - 1) / kBN;
     it.n_blocks = (kv_end + 15) >> 4;
@@ -274,11 +283,14 @@ __device__ __forceinline__ int fetch_item(const Shared &sh, int k, Item &it) {
     const uint4 *src = sh.item_slot(k);
     const uint4 a = src[0], b = src[1], c = src[2];  // field by field: the struct stays in registers
     it.req = (int)a.x, it.qrow = (int)a.y, it.prow = (int)a.z, it.rows_here = (int)a.w;
-    it.L = (int)b.x, it.spare = (int)b.y, it.n_tiles = (int)b.z, it.n_blocks = (int)b.w;
+    it.L = (int)b.x, it.nh = (int)b.y, it.n_tiles = (int)b.z, it.n_blocks = (int)b.w;
     it.head0 = (int)c.x, it.g = (int)c.y, it.malformed = (int)c.z, it.state = (int)c.w;
     return it.state == kItemWork ? 1 : 0;
 }
 
+// kSingles: the call has items of ONE head (a kv group with an odd number of query heads); the instantiation for even
+// groups carries none of the bookkeeping for a head that sits items out.
+template <bool kSingles>
 __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_constant__ CUtensorMap kvmap,
                                                                  const __grid_constant__ CUtensorMap qmap,
                                                                  const __grid_constant__ CUtensorMap omap,
@@ -288,7 +300,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
     if (*(volatile int *)p.abort_word) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t row_stride = (size_t)p.num_q_heads * kD;
-    const int n_items = p.q_tiles * (p.num_q_heads / 2);
+    const int n_items = p.q_tiles * head_pairs(p);
 
     extern __shared__ uint8_t smem_raw[];
     Shared sh;
@@ -319,7 +331,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         }
         mbar_init(sh.bar(DRAIN), 1);
         for (int i = 0; i < kItemRing; ++i) mbar_init(sh.bar(ITEM_READY + i), 1);
-        *sh.done_count() = 0;
+        for (int w = 0; w < 12; ++w) *sh.items_done(w) = 0;
         *sh.abort_flag() = 0;
         mbar_fence_init();
     }
@@ -392,7 +404,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         tiles_issued = t;
     } else if (warp == 3) {
         // =========================== item scheduler + TMA producer of the Q tiles ===========================
-        int n = 0;       // well-formed items whose Q tiles were requested so far
+        int nq[2] = {0, 0};  // Q tiles of head A / B requested so far (an item with one head has no tile for B)
         int posted = 0;  // item numbers posted so far
         bool ok = true, drained = false;
         int *counter = p.abort_word + 1;  // next item number of the launch (cleared by the launcher with the abort word)
@@ -401,11 +413,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         auto post_until = [&](int upto) -> bool {
             while (posted <= upto && !drained) {
                 if (posted >= kItemRing) {  // the ring slot is free once the 8 softmax and 4 write-out warps are through with item posted - kItemRing
-                    const int need = 12 * (posted - kItemRing + 1);
+                    const int need = posted - kItemRing + 1;
                     const uint64_t t0 = global_timer_ns();
                     bool got = false;
                     for (uint32_t i = 0; !got; ++i) {
-                        got = *(volatile int *)sh.done_count() >= need;
+                        got = __all_sync(0xffffffffu, lane >= 12 || *sh.items_done(lane) >= need);
                         if (!got) __nanosleep(100);  // nothing urgent: leave the issue slots to the softmax warp next door
                         if (!got && (i & 31u) == 31u) {
                             if (*sh.abort_flag()) return false;
@@ -420,13 +432,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 if (lane == 0) m = atomicAdd(counter, 1);
                 m = __shfl_sync(0xffffffffu, m, 0);
                 Item it;
-                it.req = it.qrow = it.prow = it.rows_here = it.L = it.spare = it.n_tiles = it.n_blocks = it.head0 = it.g = it.malformed = 0;
+                it.req = it.qrow = it.prow = it.rows_here = it.L = it.nh = it.n_tiles = it.n_blocks = it.head0 = it.g = it.malformed = 0;
                 if (m >= n_items || !decode_item(p, m, it)) it.state = kItemEnd;  // the end marker is posted once; nobody reads past it
                 drained = it.state == kItemEnd;
                 if (lane == 0) {
                     uint4 *dst = sh.item_slot(posted);
                     dst[0] = make_uint4((unsigned)it.req, (unsigned)it.qrow, (unsigned)it.prow, (unsigned)it.rows_here);
-                    dst[1] = make_uint4((unsigned)it.L, (unsigned)it.spare, (unsigned)it.n_tiles, (unsigned)it.n_blocks);
+                    dst[1] = make_uint4((unsigned)it.L, (unsigned)it.nh, (unsigned)it.n_tiles, (unsigned)it.n_blocks);
                     dst[2] = make_uint4((unsigned)it.head0, (unsigned)it.g, (unsigned)it.malformed, (unsigned)it.state);
                     __threadfence_block();
                     mbar_arrive(sh.bar(ITEM_READY + posted % kItemRing));
@@ -443,8 +455,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             if (it.malformed) continue;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
-                // the previous item's last QK^T of this head has read the tile
-                if (n > 0 && !wait_warp(sh, Q_EMPTY + x, (uint32_t)((n - 1) & 1))) {
+                if (kSingles && x >= it.nh) break;
+                // the last QK^T of this head's previous item has read the tile
+                if (nq[x] > 0 && !wait_warp(sh, Q_EMPTY + x, (uint32_t)((nq[x] - 1) & 1))) {
                     ok = false;
                     break;
                 }
@@ -453,10 +466,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 if (lane < 2)  // rows past the end of the query tensor read as zero; rows past the request's chunk are never written out
                     tma_load_3d(sh.base + kOffQ + x * kTileBytes + lane * kHalfBytes, &qmap, 64 * lane, it.head0 + x, it.qrow,
                                 sh.bar(Q_FULL + x));
+                ++nq[x];
             }
-            if (ok) ++n;
         }
-        tiles_issued = n;
+        tiles_issued = (nq[0] << 16) | nq[1];
     } else {
         // =========================== MMA issuer ===========================
         // descriptor low words of the tile origins; stepping inside a tile adds a compile-time constant
@@ -479,11 +492,14 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         // not change inside it; the values it would do that for pass through an empty asm statement.)
         int k_item = 0;
         bool list_ok = true, list_end = false;
-        int cur_tiles = 1, nxt_tiles = 0;  // all this warp needs of an item: its number of key tiles
+        int cur_tiles = 1, nxt_tiles = 0;  // all this warp needs of an item: its number of key tiles ...
+        int cur_heads = 0, nxt_heads = 0;  // ... and of query heads (2, or 1 for the odd head of an odd kv group)
         bool have_nxt = false;
         int t = 0;   // key tiles whose QK^T (both heads) has been issued: the next QK^T reads K stage t % kStages
         int tv = 0;  // key tiles whose PV has been issued
-        int n = 0;   // items whose first QK^T has been issued
+        // Head B sits out the items that have one head, so the barriers of a head count that head's own tiles and items:
+        int tvh[2] = {0, 0};  // key tiles of head x whose PV has been issued (P_PART, P_READY)
+        int nit[2] = {0, 0};  // items of head x whose first QK^T has been issued (Q_FULL, O_FREE)
         int primed = 0;  // 0 while the "current item" is the empty one in front of the list
         bool ok = true;
         while (ok) {
@@ -495,10 +511,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 else if (st == 0) list_end = true;
                 else have_nxt = !it.malformed;
                 nxt_tiles = it.n_tiles;
+                nxt_heads = it.nh;
             }
             if (!list_ok || (!primed && !have_nxt)) break;
-            int have_next = have_nxt ? 1 : 0, n_now = n, pv = primed;
-            asm volatile("" : "+r"(have_next), "+r"(n_now), "+r"(pv));
+            int have_next = have_nxt ? 1 : 0, pv = primed, heads_now = kSingles ? cur_heads : 2, heads_next = kSingles ? nxt_heads : 2;
+            asm volatile("" : "+r"(have_next), "+r"(pv));
+            if (kSingles) asm volatile("" : "+r"(heads_now), "+r"(heads_next));
 #pragma unroll 1
             for (int j = 0; j < cur_tiles && ok; ++j) {
                 const int s = tv % kStages;
@@ -509,38 +527,52 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 // that tile is the last one of its item: its QK^T is the last reader of the item's Q tile
                 const bool next_closes = new_item ? nxt_tiles == 1 : j + 2 == cur_tiles;
                 if (pv) ok = wait_warp(sh, V_FULL + s, (uint32_t)((tv / kStages) & 1));
+                const int heads_of_next_tile = last ? heads_next : heads_now;  // heads that take part in the QK^T of the next tile
+                const int tv_pre = tvh[0], nit_pre = nit[0];  // (without single-head items both heads count alike: one set of counters)
 #pragma unroll
                 for (int x = 0; x < 2 && ok; ++x) {
-                    if (pv) {
-                        // O_x still holds the previous item's result until its write-out has read it
-                        if (j == 0 && n_now > 1) ok = wait_warp(sh, O_FREE + x, (uint32_t)((n_now - 2) & 1));
-                        if (ok) ok = wait_warp(sh, P_PART + x, (uint32_t)(tv & 1));
+                    const bool pv_x = pv && x < heads_now;                 // head x has a PV on this tile
+                    const bool more_x = more && x < heads_of_next_tile;    // ... and a QK^T on the next one
+                    const bool new_x = new_item && more_x;                 // which opens an item of head x
+                    if (!pv_x && !more_x) continue;
+                    const int tvx = kSingles ? tvh[x] : tv_pre, nix = kSingles ? nit[x] : nit_pre;
+                    if (pv_x) {
+                        // O_x still holds the result of head x's previous item until the write-out warps have read it
+                        if (j == 0 && nix > 1) ok = wait_warp(sh, O_FREE + x, (uint32_t)((nix - 2) & 1));
+                        if (ok) ok = wait_warp(sh, P_PART + x, (uint32_t)(tvx & 1));
                         if (!ok) break;
                         fence_after();
                         issue_pv(x, s, j > 0, 0, kPartSteps);  // keys 0..95 while the softmax warps finish the rest
-                        ok = wait_warp(sh, P_READY + x, (uint32_t)(tv & 1));
+                        ok = wait_warp(sh, P_READY + x, (uint32_t)(tvx & 1));
                         if (!ok) break;
                     }
-                    if (more) {
+                    if (more_x) {
+                        // Head x comes back after sitting out an item: the commit below will be a completion of S_READY_x
+                        // of its own, right behind the one that said "O_x complete".  The write-out warps must have seen
+                        // that one first (a phase parity cannot tell "not yet" from "two completions ago"), and they have
+                        // once they have handed O_x back.  (Without a gap the two are one completion, and the next one
+                        // needs a PV that waits for O_FREE anyway.)
+                        if (kSingles && new_x && !pv_x && nix > 0) ok = wait_warp(sh, O_FREE + x, (uint32_t)((nix - 1) & 1));
                         // a new item: its Q tile of head x must have landed; head A also checks the K tile
-                        if (new_item) ok = wait_warp(sh, Q_FULL + x, (uint32_t)(n_now & 1));
+                        if (ok && new_x) ok = wait_warp(sh, Q_FULL + x, (uint32_t)(nix & 1));
                         if (ok && x == 0) ok = wait_warp(sh, K_FULL + s1, (uint32_t)((t / kStages) & 1));
                         if (!ok) break;
                     }
                     fence_after();
                     // The rest of the step in one go, by one elected lane: the last quarter of PV, QK^T of the next tile, and
                     // the commits (this is the stretch between "P is there" and "the next scores are there" on every
-                    // head's critical chain, so it is as few instructions as it can be).
+                    // head's critical chain, so it is as few instructions as it can be).  A K/V stage goes back to its
+                    // producer with the commit of the last head that uses it.
                     if (elect_one()) {
                         const uint64_t hi = (uint64_t)kDescHi << 32;
-                        if (pv) {
+                        if (pv_x) {
                             const uint64_t v_desc = hi | (v_lo0 + (uint32_t)s * (kTileBytes >> 4));
                             const uint32_t d = tmem + col_o(x), a = tmem + col_s(x);
 #pragma unroll
                             for (int k = kPartSteps; k < kBN / 16; ++k) mma_ts(d, a + 8 * k, v_desc + ((k * 2048) >> 4), kIdescPV, 1u);
-                            if (x == 1) mma_commit_one(sh.bar(V_EMPTY + s));
+                            if (x == heads_now - 1) mma_commit_one(sh.bar(V_EMPTY + s));
                         }
-                        if (more) {
+                        if (more_x) {
                             const uint64_t k_desc = hi | (k_lo0 + (uint32_t)s1 * (kTileBytes >> 4)), q_desc = hi | (q_lo0 + (uint32_t)x * (kTileBytes >> 4));
                             const uint32_t d = tmem + col_s(x);
 #pragma unroll
@@ -549,19 +581,23 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                                 mma_ss(d, q_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
                             }
                             if (next_closes) mma_commit_one(sh.bar(Q_EMPTY + x));
-                            if (x == 1) mma_commit_one(sh.bar(K_EMPTY + s1));
+                            if (x == heads_of_next_tile - 1) mma_commit_one(sh.bar(K_EMPTY + s1));
                         }
-                        mma_commit_one(sh.bar(S_READY + x));  // scores of the next tile, and (after an item's last tile) O_x complete
+                        // scores of head x's next tile and / or (after the last tile of an item of head x) O_x complete: when
+                        // head x sits out the next item these are two commits, one here and one when it comes back
+                        mma_commit_one(sh.bar(S_READY + x));
                     }
                     __syncwarp();
+                    if (pv_x && (kSingles || x == 0)) ++tvh[x];
+                    if (new_x && (kSingles || x == 0)) ++nit[x];
                 }
                 if (!ok) break;
                 if (pv) ++tv;
                 if (more) ++t;
-                if (new_item) ++n;
             }
             if (!ok || !have_nxt) break;
             cur_tiles = nxt_tiles;
+            cur_heads = nxt_heads;
             primed = 1;
         }
         // every MMA this thread issued must be finished before TMEM is released
@@ -581,29 +617,54 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         // S_READY_x completes once per key tile of the CTA (all items), plus once after the very last PV: completion
         // number t carries the scores of key tile t, and for the first tile of an item also "the previous item's O_x is
         // complete", which is what the write-out warps wait for.
-        int t = 0;       // key tiles processed so far (all items)
-        int n_done = 0;  // well-formed items finished so far
+        int t = 0;       // key tiles of the CTA so far (all well-formed items: K/V stages and the mask ring count these)
+        int c = 0;       // completions of S_READY_x so far: one per key tile of this head, one more each time the head
+                         // sat out an item (its last PV and its next first QK^T are then committed separately)
+        bool in_run = false;  // the previous well-formed item had this head
+        bool came_back = false;  // ... and it sat out at least one item since
+        int n_done = 0;  // items of this head finished so far
         bool ok = true;
-        auto item_done = [&]() {  // this warp is through with the item: its slot in the ring may be reused
+        int k = 0;
+        auto item_done = [&]() {  // this warp is through with the CTA's k-th item: it will not read its ring slot again
             __syncwarp();
             if (lane == 0) {
                 __threadfence_block();
-                atomicAdd(sh.done_count(), 1);
+                *sh.items_done(warp - 4) = k + 1;
             }
         };
-        for (int k = 0; ok; ++k) {
+        for (; ok; ++k) {
             Item it;
             if (fetch_item(sh, k, it) <= 0) break;
             if (it.malformed) {  // the write-out warps zero its rows
                 item_done();
                 continue;
             }
+            if (kSingles && x >= it.nh) {  // the odd head of an odd kv group: head B sits this item out
+                t += it.n_tiles;
+                // The head's last PV is committed on its own now ("O_x complete"), and its next first QK^T will be another
+                // completion of S_READY_x: count both.
+                if (in_run) ++c;
+                in_run = false;
+                came_back = true;
+                item_done();
+                continue;
+            }
+            if (kSingles && came_back && n_done > 0) {
+                // Back after sitting out: the wait for the scores below must not be two completions EARLY (a parity wait
+                // passes then as well, and these warps published their last P only a moment ago).  Once the write-out warps
+                // have handed back O_x of this head's previous item, "O_x complete" is through.  That wait cannot be late:
+                // the next hand-back needs the row sums of the item that starts here.
+                ok = wait_warp(sh, O_FREE + x, (uint32_t)((n_done - 1) & 1));
+                if (!ok) break;
+            }
+            came_back = false;
+            in_run = true;
             const int lim = it.prow + min(row, it.rows_here - 1);  // last key this row may see
             const int prow = it.prow, L = it.L, n_tiles = it.n_tiles;
             float m_run = -INFINITY, l_run = 0.f;
-            for (int j = 0; j < n_tiles; ++j, ++t) {
+            for (int j = 0; j < n_tiles; ++j, ++t, ++c) {
                 const int s = t % kStages;
-                ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1));
+                ok = wait_warp(sh, S_READY + x, (uint32_t)(c & 1));
                 if (!ok) break;
                 fence_after();
                 const int key0 = j * kBN;
@@ -758,8 +819,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         const uint32_t lane_base = (uint32_t)wrow0 << 16;
         uint8_t *stage0 = sh.ptr + kOffStage + (warp & 3) * 2 * kStageBytes;
         const int piece = lane & 7, sub = lane >> 3;
-        int t = 0;       // key tiles of the well-formed items so far: completion number t of S_READY_x says O_x is complete
-        int n = 0;       // well-formed items so far
+        int cA = 0, cB = 0;  // completions of S_READY_x up to "O_x of this item is complete": the head's key tiles so far, plus
+                             // one for every time it sat out an item (see the softmax role)
+        int nA = 0, nB = 0;  // items of head x so far
+        bool in_run = false; // the previous well-formed item had head B
         int buf = 0;     // staging buffer of the next half
         int tma_buf = -1;  // buffer that the most recent store handed to the TMA unit reads from
         bool ok = true;
@@ -771,16 +834,25 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 if (row < it.rows_here) {
                     uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)(it.qrow + row) * row_stride + (size_t)it.head0 * kD);
 #pragma unroll 1
-                    for (int c = 0; c < 2 * kD / 8; ++c) o[c] = make_uint4(0u, 0u, 0u, 0u);  // both heads: adjacent in a row
+                    for (int c8 = 0; c8 < (kSingles ? it.nh : 2) * kD / 8; ++c8) o[c8] = make_uint4(0u, 0u, 0u, 0u);  // the item's heads: adjacent in a row
                 }
             } else {
-                t += it.n_tiles;
                 const bool by_tma = wrow0 + 32 <= it.rows_here;
+                if (kSingles && it.nh < 2) {
+                    if (in_run) ++cB;
+                    in_run = false;
+                } else {
+                    in_run = true;
+                }
 #pragma unroll 1
-                for (int x = 0; x < 2 && ok; ++x) {
-                    ok = wait_warp(sh, L_READY + x, (uint32_t)(n & 1));
-                    if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)(t & 1));
+                for (int x = 0; x < (kSingles ? it.nh : 2) && ok; ++x) {
+                    if (x == 0) cA += it.n_tiles;
+                    else cB += it.n_tiles;
+                    ok = wait_warp(sh, L_READY + x, (uint32_t)((x == 0 ? nA : nB) & 1));
+                    if (ok) ok = wait_warp(sh, S_READY + x, (uint32_t)((x == 0 ? cA : cB) & 1));
                     if (!ok) break;
+                    if (x == 0) ++nA;
+                    else ++nB;
                     fence_after();
                     const float inv = sh.inv_l(x)[row];  // read before O_x is handed back: the softmax warps write the next item's late
                     const uint32_t t_o = tmem + lane_base + col_o(x);
@@ -835,12 +907,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                         buf ^= 1;
                     }
                 }
-                ++n;
             }
-            __syncwarp();  // this warp is through with the item: its slot in the ring may be reused
+            __syncwarp();  // this warp is through with the CTA's k-th item: it will not read its ring slot again
             if (lane == 0) {
                 __threadfence_block();
-                atomicAdd(sh.done_count(), 1);
+                *sh.items_done(warp - 4) = k + 1;
             }
         }
         if (lane == 0) bulk_wait_group_0();  // every row this warp handed to the TMA unit has been written
@@ -859,8 +930,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             const int FULL = warp == 2 ? V_FULL : K_FULL;
             for (int j = max(0, tiles_issued - kStages); j < tiles_issued; ++j)
                 (void)mbar_wait(sh.bar(FULL + j % kStages), (uint32_t)((j / kStages) & 1), 100000000ull);
-        } else if (warp == 3 && tiles_issued > 0) {
-            for (int x = 0; x < 2; ++x) (void)mbar_wait(sh.bar(Q_FULL + x), (uint32_t)((tiles_issued - 1) & 1), 100000000ull);
+        } else if (warp == 3) {
+            for (int x = 0; x < 2; ++x) {
+                const int nqx = x == 0 ? tiles_issued >> 16 : tiles_issued & 0xffff;  // (only the parity of the last load matters)
+                if (nqx > 0) (void)mbar_wait(sh.bar(Q_FULL + x), (uint32_t)((nqx - 1) & 1), 100000000ull);
+            }
         }
     }
     __syncthreads();
@@ -872,7 +946,8 @@ static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillPa
     static bool attr_set[64] = {false};
     const int dev = pool->desc.device;
     if (dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_prefill_chunk: shared-memory attribute");
         if (dev < 64) attr_set[dev] = true;
     }
@@ -880,11 +955,12 @@ static ekv_status_t launch_prefill_tc(ekv_pool *pool, int layer, const PrefillPa
     ekv_status_t st = encode_q_map(q, (uint64_t)total_rows, pool->desc.num_q_heads, kD, kBM, &qmap);
     if (st == EKV_OK) st = encode_q_map(out, (uint64_t)total_rows, pool->desc.num_q_heads, kD, 32, &omap);  // same geometry, 32-row boxes
     if (st != EKV_OK) return st;
-    const long long items = (long long)p.q_tiles * (pool->desc.num_q_heads / 2);
+    const long long items = (long long)p.q_tiles * head_pairs(p);
     const int grid = (int)(items < pool->sm_count ? items : pool->sm_count);
     cudaError_t e0 = cudaMemsetAsync(p.abort_word, 0, 2 * sizeof(int), stream);  // abort word + item counter
     if (e0 != cudaSuccess) return cuda_fail(e0, "ekv_attn_prefill_chunk: clear abort word and item counter");
-    prefill_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(pool->kv_map[layer], qmap, omap, p);
+    if (p.group % 2 == 0) prefill_tc_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(pool->kv_map[layer], qmap, omap, p);
+    else prefill_tc_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(pool->kv_map[layer], qmap, omap, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "ekv_attn_prefill_chunk: launch");
     return EKV_OK;

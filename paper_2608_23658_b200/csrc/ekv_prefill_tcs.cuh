@@ -102,7 +102,7 @@ __device__ __forceinline__ bool s_decode_item(const PrefillParams &p, int m, Ite
     it.prow = prefix + row0;
     it.rows_here = min(kBM, c_r - row0);
     it.malformed = prefix < 0 ? 1 : 0;
-    it.spare = 0;
+    it.nh = 0;
     const int kv_end = min(it.L, it.prow + it.rows_here);
     it.n_tiles = (kv_end + kBN - 1) / kBN;
     it.n_blocks = (kv_end + 15) >> 4;
@@ -112,7 +112,7 @@ __device__ __forceinline__ void s_read_item(const SShared &sh, int k, Item &it) 
     const uint4 *src = sh.item_slot(k);
     const uint4 a = src[0], b = src[1], c = src[2];
     it.req = (int)a.x, it.qrow = (int)a.y, it.prow = (int)a.z, it.rows_here = (int)a.w;
-    it.L = (int)b.x, it.spare = (int)b.y, it.n_tiles = (int)b.z, it.n_blocks = (int)b.w;
+    it.L = (int)b.x, it.nh = (int)b.y, it.n_tiles = (int)b.z, it.n_blocks = (int)b.w;
     it.head0 = (int)c.x, it.g = (int)c.y, it.malformed = (int)c.z, it.state = (int)c.w;
 }
 // 1 = an item to work on (possibly malformed), 0 = end of the list, -1 = the wait was given up
@@ -255,14 +255,14 @@ __global__ void __launch_bounds__(kSThreads, 1) prefill_tcs_kernel(const __grid_
                     bool is_end = false;
                     if (lane < n_post) {
                         Item it;
-                        it.req = it.qrow = it.prow = it.rows_here = it.L = it.spare = it.n_tiles = it.n_blocks = it.head0 = it.g = it.malformed = 0;
+                        it.req = it.qrow = it.prow = it.rows_here = it.L = it.nh = it.n_tiles = it.n_blocks = it.head0 = it.g = it.malformed = 0;
                         it.state = kItemEnd;
                         const int m = base + lane;
                         if (m >= n_items || !s_decode_item(p, m, it)) it.state = kItemEnd;
                         is_end = it.state == kItemEnd;
                         uint4 *dst = sh.item_slot(idx);
                         dst[0] = make_uint4((unsigned)it.req, (unsigned)it.qrow, (unsigned)it.prow, (unsigned)it.rows_here);
-                        dst[1] = make_uint4((unsigned)it.L, (unsigned)it.spare, (unsigned)it.n_tiles, (unsigned)it.n_blocks);
+                        dst[1] = make_uint4((unsigned)it.L, (unsigned)it.nh, (unsigned)it.n_tiles, (unsigned)it.n_blocks);
                         dst[2] = make_uint4((unsigned)it.head0, (unsigned)it.g, (unsigned)it.malformed, (unsigned)it.state);
                         __threadfence_block();
                         mbar_arrive(sh.bar(SITEM_READY + idx % kSRing));

@@ -53,7 +53,7 @@ def make_pool(shape, base_blocks, elastic_blocks=0, grown=False, layers=1):
 @pytest.fixture(params=["auto", "one_head", "two_head", "warp_mma"])
 def prefill_kernel(request):
     """Runs a prefill test once per kernel family: the library's own choice, then each family pinned through its pool
-    flag (two_head falls back to one_head on shapes it cannot take: head_dim 64, odd query groups)."""
+    flag (two_head falls back to one_head on shapes it cannot take: head_dim 64, a query group of one)."""
     _PREFILL_FLAGS.clear()
     if request.param != "auto":
         _PREFILL_FLAGS["prefill_" + request.param] = True
@@ -351,7 +351,8 @@ def test_prefill_c1_chunk_over_cached_prefix(prefill_kernel):
         case.close()
 
 
-@pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY, I.LLAMA70B, I.Shape(12, 4, 128), I.Shape(6, 2, 64)])
+@pytest.mark.parametrize("shape", [I.LLAMA8B, I.TINY, I.LLAMA70B, I.Shape(12, 4, 128), I.Shape(28, 4, 128), I.Shape(4, 4, 128),
+                                   I.Shape(6, 2, 64)])
 def test_prefill_batched_ragged_requests_match_oracle(shape, prefill_kernel):
     chunks = [(0, 1), (0, 100), (37, 64), (500, 129), (130, 300), (1000, 17)]  # (prefix, rows)
     lengths = [p + c for p, c in chunks]
@@ -373,7 +374,8 @@ def test_prefill_batched_ragged_requests_match_oracle(shape, prefill_kernel):
         case.close()
 
 
-@pytest.mark.parametrize("shape,R", [(I.LLAMA8B, 60), (I.TINY, 60), (I.LLAMA8B, 300)])
+@pytest.mark.parametrize("shape,R", [(I.LLAMA8B, 60), (I.TINY, 60), (I.LLAMA8B, 300), (I.Shape(28, 4, 128), 150), (I.Shape(20, 4, 128), 60),
+                                     (I.Shape(6, 2, 128), 300)])
 def test_prefill_many_requests_find_their_tiles(shape, R, prefill_kernel):
     """Many short requests in one call, some of them empty: every query tile must find its request (up to 256
     requests by bisection over a prefix table in the kernel parameters, more by walking cu_q_lens)."""
