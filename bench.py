@@ -238,14 +238,21 @@ def timed_loop(fn, steps, device, dist):
 
 # ----------------------------------------------------------------------------- side measurements
 
+# idle time before every timed prefill run (the sustained loop that follows each one-shot measurement has none)
+PREFILL_IDLE_S = 0.1
 
-def _time_reps(fn, device, reps, warmup=3):
-    """ms of `reps` separately timed runs of fn (CUDA events on the current stream), after `warmup` untimed runs."""
+
+def _time_reps(fn, device, reps, warmup=3, idle_s=0.0):
+    """ms of `reps` separately timed runs of fn (CUDA events on the current stream), after `warmup` untimed runs.
+    idle_s > 0: the device idles that long before every timed run, so that each one is a launch timed alone (what the
+    burst matmul peak is) and not the tail of a loop that has run the part into its power cap."""
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize(device)
     ts = []
     for _ in range(reps):
+        if idle_s > 0:
+            time.sleep(idle_s)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         fn()
@@ -255,11 +262,11 @@ def _time_reps(fn, device, reps, warmup=3):
     return ts
 
 
-def measure_prefill(device, peaks, reps=7, prompt_len=None, chunks=None):
+def measure_prefill(device, peaks, reps=7, prompt_len=None, chunks=None, shape=None, sustained=True):
     """Prefill-chunk TFLOP/s on the configs[2] prompt: 32768 tokens as four 8192-token chunks over
     cached prefixes 0/8k/16k/24k, and as one 32768-token chunk.  Median of `reps` runs, with min and max."""
     import paper_2608_23658_b200 as ekv
-    cfg, s = I.C3, I.C3.shape
+    cfg, s = I.C3, shape or I.C3.shape
     Lp = prompt_len or cfg.prompt_len
     nblk = Lp // s.block_size
     pool = ekv.Pool(num_q_heads=s.num_q_heads, num_kv_heads=s.num_kv_heads, head_dim=s.head_dim, base_blocks=nblk + 64,
@@ -285,7 +292,7 @@ def measure_prefill(device, peaks, reps=7, prompt_len=None, chunks=None):
             def run():
                 for (qq, oo, cud, cuh, sl) in calls:
                     pool.attn_prefill_chunk(0, qq, d_table, cud, cuh, sl, scale, out=oo)
-            ts = _time_reps(run, device, reps)
+            ts = _time_reps(run, device, reps, idle_s=PREFILL_IDLE_S)
             med = statistics.median(ts)
             flops = sum(I.prefill_flops(chunk, start, s) for start in range(0, Lp, chunk))
             tf = flops / (med * 1e-3) / 1e12
@@ -296,7 +303,7 @@ def measure_prefill(device, peaks, reps=7, prompt_len=None, chunks=None):
                                      "frac_of_measured_bf16": round(tf / peaks["bf16_tflops"], 4),
                                      "frac_of_measured_bf16_sustained": round(tf / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), 4),
                                      "frac_of_nominal_2250": round(tf / 2250.0, 4)}
-            if len(calls) == 1:
+            if len(calls) == 1 and sustained:
                 # the same launch back to back for about a second, clocks sampled meanwhile: the figure to hold
                 # against the sustained matmul peak, which was measured the same way
                 n_loop = max(8, int(1000.0 / med))
@@ -319,7 +326,8 @@ def measure_prefill(device, peaks, reps=7, prompt_len=None, chunks=None):
                     "frac_of_measured_bf16_sustained": round(tf_loop / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), 4),
                     "sm_mhz": clk["sm_mhz"], "reasons": clk["reasons"]}
                 time.sleep(0.5)     # let the part leave its power cap before the next measurement
-        res["workload"] = f"c3 prompt {Lp} tokens, 32/8 heads d128, causal-exact FLOPs of both contractions, median of {reps}"
+        res["workload"] = (f"c3 prompt {Lp} tokens, {s.num_q_heads}/{s.num_kv_heads} heads d{s.head_dim}, causal-exact FLOPs of both "
+                           f"contractions, median of {reps} runs with {int(PREFILL_IDLE_S * 1e3)} ms of idle before each")
         return res
     finally:
         pool.close()
@@ -867,6 +875,8 @@ def main(argv=None):
         # of the line holds prefill, mixed step, long-context decode, write and the CPU baseline.
         torch.cuda.empty_cache()
         pf = measure_prefill(device, peaks)
+        # the same prompt on the head layout of the paper's model (28 query / 4 kv heads: groups of 7, an odd number)
+        pf_g7 = measure_prefill(device, peaks, reps=5, chunks=(I.C3.prompt_len,), shape=I.Shape(28, 4, 128), sustained=False)
         torch.cuda.empty_cache()
         pf_short = measure_prefill_short(device, peaks)
         torch.cuda.empty_cache()
@@ -884,13 +894,18 @@ def main(argv=None):
         line["write_kv"] = wkv
         line["mixed_step"] = mixed
         line["prefill_short"] = pf_short
+        g7 = pf_g7[f"chunk_{I.C3.prompt_len}"]
+        line["prefill_group_of_7"] = {"ms": g7["ms"], "ms_min": g7["ms_min"], "tflops": g7["tflops"],
+                                      "frac_of_measured_bf16": g7["frac_of_measured_bf16"], "workload": pf_g7["workload"]}
         line["prefill"] = pf
         one_shot = pf["chunk_32768"]
         line["roofline_prefill"] = {
             "bound": "tensor", "kernel": "prefill_tc_kernel", "achieved": one_shot["tflops"], "peak": peaks["bf16_tflops"],
             "unit": "TFLOP/s", "frac": one_shot["frac_of_measured_bf16"], "peak_kind": f"{peaks_kind} cuBLAS bf16 burst",
             "frac_of_sustained_peak": one_shot["frac_of_measured_bf16_sustained"], "best_of_runs": one_shot["tflops_best"],
-            "launch_ms": one_shot["ms"], "workload": "c3 prompt, one 32768-token chunk, median of 7 launches",
+            "launch_ms": one_shot["ms"],
+            "workload": f"c3 prompt, one 32768-token chunk, median of 7 launches timed alone ({int(PREFILL_IDLE_S * 1e3)} ms of idle before each); "
+                        "sustained_loop = the same launch back to back for a second",
             "chunked_4x8192_tflops": pf["chunk_8192"]["tflops"], "sustained_loop": one_shot.get("sustained"),
             "traffic": None}
         one, nbytes, sample, cores = oracle_decode_sample(cfg)
