@@ -235,7 +235,7 @@ struct Item {
     int L, n_tiles, n_blocks;  // keys of the request; key tiles / blocks any row of this tile may see
     int head0, g;   // first of the two query heads; their kv-head
     int nh;         // query heads of the item: 2, or 1 for the odd head of a kv group with an odd number of query heads
-    int malformed;  // seq_len shorter than the chunk: rows are zero-filled, nothing is loaded or multiplied
+    int malformed;  // seq_len shorter than the chunk: the scheduler zero-fills the rows itself and never posts the item
     int state;      // kItemWork, or kItemEnd: the list of this CTA ends here
 };
 static constexpr int kItemWork = 1, kItemEnd = 2;
@@ -276,7 +276,7 @@ __device__ __forceinline__ bool decode_item(const PrefillParams &p, int m, Item 
 }
 
 // The CTA's k-th item as posted by the scheduler.  Returns 1 for an item to work on, 0 at the end of the list (or for
-// an item that names no request), -1 if the wait was given up.  A malformed item still counts as 1.
+// an item that names no request), -1 if the wait was given up.
 __device__ __forceinline__ int fetch_item(const Shared &sh, int k, Item &it) {
     const bool got = wait_warp(sh, ITEM_READY + k % kItemRing, (uint32_t)((k / kItemRing) & 1));
     if (!got) return -1;
@@ -361,7 +361,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         for (int k = 0; ok; ++k) {
             Item it;
             if (fetch_item(sh, k, it) <= 0) break;
-            if (it.malformed) continue;
             const int *bt = p.block_tables + (size_t)it.req * p.max_blocks;
             auto load_id = [&](int j) {  // lane l: id of block 8j + l%8 (-1 past the end, -2 invalid)
                 int id = -1;
@@ -435,6 +434,18 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 it.req = it.qrow = it.prow = it.rows_here = it.L = it.nh = it.n_tiles = it.n_blocks = it.head0 = it.g = it.malformed = 0;
                 if (m >= n_items || !decode_item(p, m, it)) it.state = kItemEnd;  // the end marker is posted once; nobody reads past it
                 drained = it.state == kItemEnd;
+                if (!drained && it.malformed) {
+                    // A request with fewer keys than query rows: its rows are zero-filled here and the item is not posted.
+                    // (Posted and skipped by every role it tied the ring in a knot: "O of item i is complete" comes with the
+                    // first QK^T of the next item that has work, whose Q tile this warp loads only after it has posted one
+                    // item more, for which it needs the slot of an item three back -- item i again, if two such items lie in
+                    // between.)
+                    if (lane == 0) atomicOr(p.status, EKV_DEV_FLAG_OOB);
+                    for (int r = 0; r < it.rows_here; ++r)
+                        if (lane < 16 * it.nh)  // 256 bytes per head and row; the item's heads are adjacent in a row
+                            reinterpret_cast<uint4 *>(p.out + (size_t)(it.qrow + r) * row_stride + (size_t)it.head0 * kD)[lane] = make_uint4(0u, 0u, 0u, 0u);
+                    continue;
+                }
                 if (lane == 0) {
                     uint4 *dst = sh.item_slot(posted);
                     dst[0] = make_uint4((unsigned)it.req, (unsigned)it.qrow, (unsigned)it.prow, (unsigned)it.rows_here);
@@ -452,7 +463,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
             if (!ok || k >= posted) break;
             Item it;
             if (fetch_item(sh, k, it) <= 0) break;  // posted by this warp: the wait passes at once
-            if (it.malformed) continue;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 if (kSingles && x >= it.nh) break;
@@ -509,7 +519,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
                 const int st = fetch_item(sh, k_item++, it);
                 if (st < 0) list_ok = false;
                 else if (st == 0) list_end = true;
-                else have_nxt = !it.malformed;
+                else have_nxt = true;
                 nxt_tiles = it.n_tiles;
                 nxt_heads = it.nh;
             }
@@ -635,10 +645,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         for (; ok; ++k) {
             Item it;
             if (fetch_item(sh, k, it) <= 0) break;
-            if (it.malformed) {  // the write-out warps zero its rows
-                item_done();
-                continue;
-            }
             if (kSingles && x >= it.nh) {  // the odd head of an odd kv group: head B sits this item out
                 t += it.n_tiles;
                 // The head's last PV is committed on its own now ("O_x complete"), and its next first QK^T will be another
@@ -829,14 +835,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(const __grid_co
         for (int k = 0; ok; ++k) {
             Item it;
             if (fetch_item(sh, k, it) <= 0) break;
-            if (it.malformed) {  // seq_len shorter than the chunk: zero rows, latch
-                if (threadIdx.x == 384) atomicOr(p.status, EKV_DEV_FLAG_OOB);
-                if (row < it.rows_here) {
-                    uint4 *o = reinterpret_cast<uint4 *>(p.out + (size_t)(it.qrow + row) * row_stride + (size_t)it.head0 * kD);
-#pragma unroll 1
-                    for (int c8 = 0; c8 < (kSingles ? it.nh : 2) * kD / 8; ++c8) o[c8] = make_uint4(0u, 0u, 0u, 0u);  // the item's heads: adjacent in a row
-                }
-            } else {
+            {
                 const bool by_tma = wrow0 + 32 <= it.rows_here;
                 if (kSingles && it.nh < 2) {
                     if (in_run) ++cB;

@@ -44,7 +44,7 @@ static_assert(kSOffMask + 32 <= kSOffItems, "barrier area");
 // the number of warps launched).
 static constexpr int kSThreads = 384, kSLaunchRegs = 168;
 static_assert(128 * 72 + 256 * 216 <= kSLaunchRegs * kSThreads && kSLaunchRegs * kSThreads <= 65536, "register split of the two-slot kernel");
-static constexpr int kSSmemBytes = kOffBar + kSOffItems + 64 * kSRing + 1024;  // + alignment slack
+static constexpr int kSSmemBytes = kOffBar + kSOffItems + 64 * kSRing + 32 + 1024;  // + per-warp progress, + alignment slack
 static_assert(kSSmemBytes <= 232448, "shared memory of one CTA");
 
 struct SShared {
@@ -53,10 +53,12 @@ struct SShared {
     __device__ __forceinline__ uint32_t bar(int i) const { return base + kOffBar + 8 * i; }
     __device__ __forceinline__ volatile int *abort_flag() const { return (volatile int *)(ptr + kOffBar + kSOffFlags); }
     __device__ __forceinline__ uint32_t *tmem_slot() const { return (uint32_t *)(ptr + kOffBar + kSOffFlags + 4); }
-    // Finished items are COUNTED (4 warps per item and slot), not signalled on an mbarrier: the scheduler looks at the
-    // count only when it needs a ring slot back, possibly several items later, and a phase parity cannot tell "not yet"
-    // from "two phases ago".
-    __device__ __forceinline__ int *done_count(int x) const { return (int *)(ptr + kOffBar + kSOffFlags + 8 + 4 * x); }
+    // Finished items are COUNTED, not signalled on an mbarrier: the scheduler looks only when it needs a ring slot back,
+    // possibly several items later, and a phase parity cannot tell "not yet" from "two phases ago".  Every softmax warp
+    // keeps its own count (items of its slot it is through with) and the scheduler takes the minimum of a slot's four: in
+    // a sum the lead of three warps could pay for the one that lags (they are not tied to each other on items that have
+    // no tiles).
+    __device__ __forceinline__ volatile int *items_done(int x) const { return (volatile int *)(ptr + kOffBar + kSOffItems + 64 * kSRing) + 4 * x; }
     // per slot a ring of 4 masks of key blocks whose shared-memory rows hold stand-in data
     __device__ __forceinline__ volatile int *bad_mask(int x, int tile) const {
         return (volatile int *)(ptr + kOffBar + kSOffMask + 16 * x + 4 * (tile & 3));
@@ -153,7 +155,7 @@ __global__ void __launch_bounds__(kSThreads, 1) prefill_tcs_kernel(const __grid_
             mbar_init(sh.bar(SP_READY + x), 128);
             mbar_init(sh.bar(SP_PART + x), 128);
             mbar_init(sh.bar(SO_FREE + x), 4);
-            *sh.done_count(x) = 0;
+            for (int w = 0; w < 4; ++w) sh.items_done(x)[w] = 0;
         }
         mbar_init(sh.bar(SDRAIN), 1);
         for (int i = 0; i < kSRing; ++i) mbar_init(sh.bar(SITEM_READY + i), 1);
@@ -246,7 +248,8 @@ __global__ void __launch_bounds__(kSThreads, 1) prefill_tcs_kernel(const __grid_
             if (ends < 2) {
                 const int idx = posted + lane;
                 const bool can = lane < 4 && idx < min(qk[0], qk[1]) + kSRing - 2 &&
-                                 (idx < kSRing || *(volatile int *)sh.done_count(idx & 1) >= 4 * (((idx - kSRing) >> 1) + 1));
+                                 (idx < kSRing || min(min(sh.items_done(idx & 1)[0], sh.items_done(idx & 1)[1]),
+                                                      min(sh.items_done(idx & 1)[2], sh.items_done(idx & 1)[3])) >= ((idx - kSRing) >> 1) + 1);
                 const int n_post = __ffs((int)~__ballot_sync(0xffffffffu, can)) - 1;  // leading lanes that can
                 if (n_post > 0) {
                     int base = 0;
@@ -425,14 +428,15 @@ __global__ void __launch_bounds__(kSThreads, 1) prefill_tcs_kernel(const __grid_
         // t + n belongs to key tile t of the slot when n items were finished before it.
         int t = 0, n = 0;
         bool ok = true;
-        auto item_done = [&]() {  // this warp will not read the item's ring slot again
+        int k = x;
+        auto item_done = [&]() {  // this warp will not read the ring slot of the CTA's k-th item again
             __syncwarp();
             if (lane == 0) {
                 __threadfence_block();
-                atomicAdd(sh.done_count(x), 1);
+                sh.items_done(x)[warp & 3] = (k >> 1) + 1;
             }
         };
-        for (int k = x; ok; k += 2) {
+        for (; ok; k += 2) {
             Item it;
             if (s_fetch_item(sh, k, it, p.status, p.abort_word) <= 0) break;
             if (it.malformed) {  // zero rows, latch

@@ -602,6 +602,45 @@ def test_prefill_request_with_fewer_keys_than_rows_is_zeroed_and_latched(prefill
         case.close()
 
 
+@pytest.mark.parametrize("shape", [I.LLAMA8B, I.Shape(28, 4, 128)])
+def test_prefill_many_invalid_requests_among_valid_ones(shape, prefill_kernel):
+    """A batch of short requests in which about a third have fewer keys than rows, often several in a row: the
+    persistent kernels walk lists in which items without work follow each other, and must neither stall nor mix up
+    the others (rows of invalid requests are zeros, the rest matches the oracle, EKV_ERR_BLOCK_OOB is latched)."""
+    R = 400
+    rows = I.uniform_ints(111, 1, R, 2, 140)
+    prefix = I.uniform_ints(111, 2, R, 0, 40)
+    lengths = rows + prefix
+    case = Case(shape, lengths.tolist(), int(I.blocks_for(lengths, 16).sum()) + 5, 112)
+    try:
+        cu = torch.cat([torch.zeros(1, dtype=torch.int64), torch.cumsum(rows, 0)]).to(torch.int32)
+        q = rand_q(113, int(cu[-1]), shape)
+        scale = 1 / math.sqrt(shape.head_dim)
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q, case.tables,
+                                         cu, case.lengths, scale)
+        pick = I.uniform_ints(111, 3, R, 0, 99)
+        invalid = [r for r in range(R) if int(pick[r]) < 35 or 100 <= r < 112]       # a third of them, and a run of twelve
+        short = case.d_lengths.clone()
+        for r in invalid:
+            short[r] = int(rows[r]) - 1
+        out = torch.full((int(cu[-1]), shape.num_q_heads, shape.head_dim), 7.0, dtype=torch.bfloat16, device=DEV)
+        for _ in range(2):
+            case.pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, short, scale, out=out)
+        torch.cuda.synchronize()
+        assert case.pool.poll_status() == ekv.Status.ERR_BLOCK_OOB
+        got = out.float().cpu().numpy().astype(np.float64)
+        bad = set(invalid)
+        for r in range(R):
+            a, b = int(cu[r]), int(cu[r + 1])
+            if r in bad:
+                assert not got[a:b].any(), f"request {r}: rows of an invalid request must be zeros"
+            else:
+                err = np.abs(got[a:b] - want[a:b])
+                assert err.max() <= MAX_ABS, f"request {r}: max-abs {err.max():.4g}"
+    finally:
+        case.close()
+
+
 def test_prefill_calls_in_flight_on_two_streams_keep_their_own_work_lists():
     """Two chunked-prefill calls of one pool running at the same time (two streams, different requests): the persistent
     kernel hands out its work items from a counter in device memory, and every launch must have its own."""
