@@ -641,6 +641,44 @@ def test_prefill_many_invalid_requests_among_valid_ones(shape, prefill_kernel):
         case.close()
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_prefill_random_batches_match_oracle_and_repeat_bit_for_bit(seed):
+    """Seeded random batches (head layout, number of requests, chunk and prefix lengths, empty and invalid requests):
+    the library's own kernel choice against the oracle, and the same call twice must give the same bits (a race between
+    the roles of a persistent CTA shows up as a difference between runs long before it shows up as a wrong value)."""
+    hq, hkv = [(32, 8), (28, 4), (12, 4), (8, 8), (20, 4), (64, 8), (6, 2), (16, 8)][seed]
+    shape = I.Shape(hq, hkv, 128)
+    R = [1, 3, 17, 40, 90, 150, 60, 25][seed]
+    rows = I.uniform_ints(500 + seed, 1, R, 0, [900, 400, 300, 200, 140, 60, 129, 260][seed])
+    prefix = I.uniform_ints(500 + seed, 2, R, 0, [1500, 700, 300, 200, 60, 130, 10, 400][seed])
+    rows[0] = max(int(rows[0]), 1)
+    lengths = rows + prefix
+    case = Case(shape, lengths.tolist(), int(I.blocks_for(lengths, 16).sum()) + 3, 600 + seed)
+    try:
+        cu = torch.cat([torch.zeros(1, dtype=torch.int64), torch.cumsum(rows, 0)]).to(torch.int32)
+        q = rand_q(700 + seed, int(cu[-1]), shape)
+        scale = 1 / math.sqrt(shape.head_dim)
+        pick = I.uniform_ints(500 + seed, 3, R, 0, 99)
+        invalid = [r for r in range(1, R) if int(pick[r]) < 12 and int(rows[r]) > 1]
+        seq = case.d_lengths.clone()
+        for r in invalid:
+            seq[r] = int(rows[r]) - 1
+        outs = [case.pool.attn_prefill_chunk(0, q.to(DEV), case.d_tables, cu.to(DEV), cu, seq, scale).clone() for _ in range(3)]
+        torch.cuda.synchronize()
+        assert case.pool.poll_status() == (ekv.Status.ERR_BLOCK_OOB if invalid else ekv.Status.OK)
+        assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+        want = oracle.attn_prefill_chunk(case.host, shape.num_q_heads, shape.num_kv_heads, 16, shape.head_dim, q, case.tables,
+                                         cu, case.lengths, scale)
+        got = outs[0].float().cpu().numpy().astype(np.float64)
+        for r in invalid:
+            a, b = int(cu[r]), int(cu[r + 1])
+            assert not got[a:b].any()
+            want[a:b] = 0.0
+        check_close(outs[0], want, f"random batch {seed}, {hq}q/{hkv}kv, {R} requests")
+    finally:
+        case.close()
+
+
 def test_prefill_calls_in_flight_on_two_streams_keep_their_own_work_lists():
     """Two chunked-prefill calls of one pool running at the same time (two streams, different requests): the persistent
     kernel hands out its work items from a counter in device memory, and every launch must have its own."""
